@@ -1,0 +1,178 @@
+/*
+ * pvlm.h - C ABI of the per-step verify / prune / accept hot path of a
+ * draft-then-verify (speculative decoding) loop for Video-LLMs, for NVIDIA
+ * B200 (sm_100a).
+ *
+ * Conventions for every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless the
+ *     field says "host".  The library never frees or retains caller memory.
+ *   - Calls are asynchronous on the CUDA stream passed as `void *stream`
+ *     (a cudaStream_t; NULL = default stream).  The library never
+ *     synchronises the stream or the device.
+ *   - Scratch memory is caller-provided: `workspace` must hold at least the
+ *     number of bytes the matching *_workspace_bytes query returns for the
+ *     same parameter struct, and be 256-byte aligned.  Workspace contents are
+ *     undefined before and after a call.  Two calls that may overlap on the
+ *     GPU need distinct workspaces.
+ *   - Outputs are overwritten, never accumulated; inputs are never modified.
+ *   - Argument errors are detected on the host before anything is launched
+ *     and reported through the return value; no device-side trap exists.
+ *   - Results are run-to-run deterministic (no floating-point atomics).
+ *   - bf16 tensors are passed as `void *` (2 bytes per element).
+ *   - All base pointers of bf16 / fp32 tensors must be 16-byte aligned and
+ *     bf16 strides must be multiples of 8 elements.
+ */
+#ifndef PVLM_H
+#define PVLM_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int pvlm_status;
+enum {
+  PVLM_OK = 0,
+  PVLM_ERR_INVALID_ARG = 1, /* NULL where data is required, negative size, bad stride or alignment */
+  PVLM_ERR_UNSUPPORTED = 2, /* shape outside the compiled set (see each call) */
+  PVLM_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned or too small */
+  PVLM_ERR_CUDA = 4         /* a launch failed; see pvlm_last_cuda_error() */
+};
+
+/* Human-readable name of a status code (static storage). */
+const char *pvlm_status_string(pvlm_status s);
+/* cudaError_t (as int) of the most recent failed launch on this host thread, 0 if none. */
+int pvlm_last_cuda_error(void);
+/* Library version: major * 1000 + minor. */
+int pvlm_version(void);
+
+/* ------------------------------------------------------------------------
+ * Window-verify grouped-query attention with attention-mass emission.
+ *
+ * The target model verifies the gamma drafted tokens in one parallel pass
+ * over the full multimodal context (paper Sec. 2.2; Sec. 4.2, Stage II).
+ * Per layer: window row r (0 <= r < R, R = gamma + 1) of query head h attends
+ * keys j in [0, n_ctx + r] of KV head floor(h / (Hq / Hkv)):
+ *     s_j = softmax_scale * <q[r,h,:], k[j,g,:]>,  P = softmax_j(s),
+ *     o[r,h,:] = sum_j P_j v[j,g,:],  lse[h,r] = log sum_j exp(s_j).
+ * The attention mass of key j is sum over all h and r of P_j: the
+ * attention-score signal that attention-guided pruning ranks visual tokens
+ * by (paper Sec. 3, Challenge 2), which a block-wise attention kernel does
+ * not otherwise expose.
+ *
+ * T = n_ctx + R rows of k and v are read per layer: the committed context
+ * followed by the window's own rows.  n_layers > 1 batches independent
+ * layers into one launch.
+ *
+ * Supported: D in {64, 128}; Hq % Hkv == 0; 1 <= R; (Hq / Hkv) * R <= 128;
+ * n_ctx >= 0; n_layers >= 1.  Anything else returns PVLM_ERR_UNSUPPORTED.
+ * bf16 inputs, fp32 accumulation; o is rounded to bf16 once at the end.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+  const void *q;        /* bf16 [n_layers][R][Hq][D], layer stride q_layer_stride            */
+  const void *k;        /* bf16 [n_layers][T][Hkv][D], strides below                          */
+  const void *v;        /* bf16, same layout and strides as k                                  */
+  void *o;              /* bf16 [n_layers][R][Hq][D], same layer stride as q                   */
+  float *lse;           /* fp32 [n_layers][Hq][R] natural-log lse; nullable                    */
+  float *mass;          /* fp32 [n_layers][T], layer stride mass_layer_stride; nullable =>
+                           the mass pass is skipped for the whole call                         */
+  int n_layers, R, Hq, Hkv, D, n_ctx;
+  long long q_layer_stride;    /* elements */
+  long long kv_layer_stride;   /* elements */
+  long long kv_token_stride;   /* elements, >= Hkv * kv_head_stride                            */
+  long long kv_head_stride;    /* elements, >= D                                               */
+  long long mass_layer_stride; /* elements, >= T                                               */
+  float softmax_scale;         /* 0 => 1/sqrt(D)                                               */
+  void *workspace;
+  size_t workspace_bytes;
+} pvlm_attn_params;
+
+/* Host-only; needs no GPU.  Returns 0 if the parameters are unsupported. */
+size_t pvlm_verify_attn_workspace_bytes(const pvlm_attn_params *p);
+pvlm_status pvlm_verify_attn(const pvlm_attn_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
+ * UV-Prune: debiased score, Top-K selection, gather into the draft cache.
+ *
+ * score_i = mass_cur[vis_start + i] - mass_ref[vis_start + i] for the m
+ * visual tokens: the layer-to-layer variation of the relevance signal summed
+ * over layers (paper Eq. 2), which telescopes to the difference of its two
+ * end layers and cancels the layer-invariant positional part (Appendix E).
+ * One fp32 subtraction, round to nearest.  mass_ref == NULL ranks by the raw
+ * signal.  The k largest scores are kept (Eq. 3; k = (1 - alpha) m, Eq. 5);
+ * equal scores are kept lower index first (-0.0 == +0.0; NaN ranks below
+ * every number); kept_idx is ascending, relative to vis_start.
+ *
+ * If src_k is non-NULL the kept rows are gathered, per layer and for K and V:
+ *   dst = [ src[0, vis_start) ; src[vis_start + kept_idx[.]] ; src[vis_start + m, src_len) ]
+ * i.e. the draft context keeps the selected visual tokens and everything
+ * else (paper Sec. 4.2, Stage I: draft prefix = (V*, X_{1:n})).  Byte copy.
+ *
+ * Supported: 0 <= k <= m <= 2^24; row_bytes % 16 == 0; src/dst 16-byte aligned.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+  const float *mass_cur; /* fp32 [>= vis_start + m]                                           */
+  const float *mass_ref; /* fp32 [>= vis_start + m]; nullable                                 */
+  int vis_start, m, k;
+  int *kept_idx;         /* int32 [k] out                                                      */
+  float *score;          /* fp32 [m] out; nullable                                             */
+  const void *src_k, *src_v; /* [n_layers][src_len][row_bytes]; both NULL => select only      */
+  void *dst_k, *dst_v;       /* [n_layers][src_len - m + k][row_bytes]                         */
+  int n_layers, src_len;
+  long long row_bytes;
+  long long src_layer_stride_bytes, dst_layer_stride_bytes;
+  void *workspace;
+  size_t workspace_bytes;
+} pvlm_prune_params;
+
+size_t pvlm_uvprune_workspace_bytes(const pvlm_prune_params *p);
+pvlm_status pvlm_uvprune_select_gather(const pvlm_prune_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Vocab softmax + lossless accept / reject + residual resampling.
+ *
+ * p_t = softmax(target_logits[t] / temperature), t = 0..gamma;
+ * q_t = softmax(draft_logits[t] / temperature), t = 0..gamma-1.
+ * Drafted token x_t is accepted with probability min{1, p_t(x_t)/q_t(x_t)}
+ * (paper Sec. 2.2), evaluated as u_t * q_t(x_t) < p_t(x_t) in fp32; at the
+ * first rejection n a replacement is drawn from norm(max(0, p_n - q_n))
+ * (same section); if all gamma are accepted one token is drawn from
+ * p_gamma.  The draw is an inverse CDF in vocabulary order with uniform
+ * u_gamma: the smallest j whose cumulative weight exceeds u * total.
+ *
+ * `batch` independent sequences share gamma and V; sequence b uses
+ * target_logits + b * target_batch_stride, etc. (a batch stride of 0 lets
+ * every sequence read the same logits); small per-sequence arrays are densely
+ * packed [batch][...].  Full-probability outputs, if requested, use the same
+ * strides as the logits (so they need non-zero batch strides).
+ *
+ * Supported: 1 <= gamma <= 64; 1 <= V < 2^31; 1 <= batch <= 65535.  Rows are
+ * read with 16-byte loads when the logit base pointers are 16-byte aligned
+ * and all logit strides are multiples of 4 elements, else element by element.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+  const float *target_logits;  /* fp32 [batch][gamma+1][V]                                    */
+  const float *draft_logits;   /* fp32 [batch][gamma][V]                                      */
+  long long target_row_stride, draft_row_stride;     /* elements                               */
+  long long target_batch_stride, draft_batch_stride; /* elements                               */
+  const int *draft_tokens;     /* int32 [batch][gamma], each in [0, V)                         */
+  const float *uniforms;       /* fp32 [batch][gamma+1] in [0,1): gamma accept tests, 1 draw   */
+  int batch, gamma, V;
+  float temperature;           /* 0 or 1 => 1                                                  */
+  int *n_accept;               /* int32 [batch] out, in [0, gamma]                             */
+  int *out_tokens;             /* int32 [batch][gamma+1] out: n_accept drafts, the drawn token, then -1 */
+  float *p_tok, *q_tok;        /* fp32 [batch][gamma] out: p_t(x_t), q_t(x_t) for every t; nullable     */
+  float *lse_p, *lse_q;        /* fp32 [batch][gamma+1], [batch][gamma] out (of logits/temperature); nullable */
+  float *probs_p, *probs_q;    /* fp32 full probabilities, same strides as the logits; nullable (tests) */
+  void *workspace;
+  size_t workspace_bytes;
+} pvlm_accept_params;
+
+size_t pvlm_spec_accept_workspace_bytes(const pvlm_accept_params *p);
+pvlm_status pvlm_spec_accept(const pvlm_accept_params *p, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PVLM_H */

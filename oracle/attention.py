@@ -45,9 +45,10 @@ def verify_attn(q_bits, k_bits, v_bits, n_ctx: int, scale: float | None = None, 
     mass = np.zeros(T)
     for h in (range(Hq) if heads is None else heads):
         g = h // G
+        S = scale * (k[:, g, :] @ q[:, h, :].T)         # [T, R] scores of head h against every key
         for r in range(R):
-            vis = n_ctx + r + 1                      # keys 0 .. n_ctx + r
-            s = scale * (k[:vis, g, :] @ q[r, h, :])
+            vis = n_ctx + r + 1                          # row r sees keys 0 .. n_ctx + r
+            s = S[:vis, r]
             M = s.max()
             e = np.exp(s - M)
             Z = e.sum()

@@ -1,0 +1,266 @@
+"""Thin ctypes binding over libpvlm.so: argument marshalling only.
+
+Function names and argument meaning follow include/pvlm.h.  torch is used for
+device memory and streams; every step of the path runs in the library's CUDA
+kernels.  There is no CPU fallback: if the shared library cannot be loaded or
+built, or a tensor is not on a CUDA device, the call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import threading
+
+import torch
+
+from . import build as _build
+
+_LIB = None
+_LOCK = threading.Lock()
+
+STATUS_NAMES = {0: "PVLM_OK", 1: "PVLM_ERR_INVALID_ARG", 2: "PVLM_ERR_UNSUPPORTED",
+                3: "PVLM_ERR_WORKSPACE", 4: "PVLM_ERR_CUDA"}
+
+
+class PvlmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class AttnParams(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("o", C.c_void_p),
+                ("lse", C.c_void_p), ("mass", C.c_void_p),
+                ("n_layers", C.c_int), ("R", C.c_int), ("Hq", C.c_int), ("Hkv", C.c_int), ("D", C.c_int),
+                ("n_ctx", C.c_int),
+                ("q_layer_stride", C.c_longlong), ("kv_layer_stride", C.c_longlong),
+                ("kv_token_stride", C.c_longlong), ("kv_head_stride", C.c_longlong),
+                ("mass_layer_stride", C.c_longlong),
+                ("softmax_scale", C.c_float),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+class PruneParams(C.Structure):
+    _fields_ = [("mass_cur", C.c_void_p), ("mass_ref", C.c_void_p),
+                ("vis_start", C.c_int), ("m", C.c_int), ("k", C.c_int),
+                ("kept_idx", C.c_void_p), ("score", C.c_void_p),
+                ("src_k", C.c_void_p), ("src_v", C.c_void_p), ("dst_k", C.c_void_p), ("dst_v", C.c_void_p),
+                ("n_layers", C.c_int), ("src_len", C.c_int),
+                ("row_bytes", C.c_longlong), ("src_layer_stride_bytes", C.c_longlong),
+                ("dst_layer_stride_bytes", C.c_longlong),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+class AcceptParams(C.Structure):
+    _fields_ = [("target_logits", C.c_void_p), ("draft_logits", C.c_void_p),
+                ("target_row_stride", C.c_longlong), ("draft_row_stride", C.c_longlong),
+                ("target_batch_stride", C.c_longlong), ("draft_batch_stride", C.c_longlong),
+                ("draft_tokens", C.c_void_p), ("uniforms", C.c_void_p),
+                ("batch", C.c_int), ("gamma", C.c_int), ("V", C.c_int), ("temperature", C.c_float),
+                ("n_accept", C.c_void_p), ("out_tokens", C.c_void_p),
+                ("p_tok", C.c_void_p), ("q_tok", C.c_void_p), ("lse_p", C.c_void_p), ("lse_q", C.c_void_p),
+                ("probs_p", C.c_void_p), ("probs_q", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
+           "pvlm_verify_attn_workspace_bytes", "pvlm_verify_attn",
+           "pvlm_uvprune_workspace_bytes", "pvlm_uvprune_select_gather",
+           "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept")
+
+
+def lib() -> C.CDLL:
+    """Load (building it first if absent or stale) the C-ABI library."""
+    global _LIB
+    with _LOCK:
+        if _LIB is None:
+            path = _build.build()
+            L = C.CDLL(path)
+            L.pvlm_status_string.restype = C.c_char_p
+            L.pvlm_status_string.argtypes = [C.c_int]
+            L.pvlm_last_cuda_error.restype = C.c_int
+            L.pvlm_version.restype = C.c_int
+            for name, st in (("verify_attn", AttnParams), ("uvprune", PruneParams), ("spec_accept", AcceptParams)):
+                f = getattr(L, f"pvlm_{name}_workspace_bytes")
+                f.restype = C.c_size_t
+                f.argtypes = [C.POINTER(st)]
+            for name, st in (("pvlm_verify_attn", AttnParams), ("pvlm_uvprune_select_gather", PruneParams),
+                             ("pvlm_spec_accept", AcceptParams)):
+                f = getattr(L, name)
+                f.restype = C.c_int
+                f.argtypes = [C.POINTER(st), C.c_void_p]
+            _LIB = L
+    return _LIB
+
+
+_WS: dict = {}
+
+
+def _workspace(dev: torch.device, key: str, nbytes: int) -> torch.Tensor:
+    """A per-(device, stream, call kind) scratch buffer that only grows."""
+    k = (dev.index, torch.cuda.current_stream(dev).cuda_stream, key)
+    buf = _WS.get(k)
+    if buf is None or buf.numel() < nbytes:
+        buf = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=dev)
+        _WS[k] = buf
+    return buf
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _need_cuda(*ts):
+    for t in ts:
+        if t is not None and not t.is_cuda:
+            raise RuntimeError("pvlm: tensors must live on a CUDA device (there is no CPU path)")
+
+
+def _stream(dev):
+    return C.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
+
+
+def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None) -> AttnParams:
+    """Fill an AttnParams from torch tensors: q/o [L,R,Hq,D] or [R,Hq,D]; k/v [L,T,Hkv,D] or [T,Hkv,D]."""
+    if q.dim() == 3:
+        q, k, v, o = q[None], k[None], v[None], o[None]
+    L, R, Hq, D = q.shape
+    _, T, Hkv, _ = k.shape
+    assert T == n_ctx + R, "k/v must hold n_ctx + R rows"
+    assert q.dtype == torch.bfloat16 and k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16
+    assert q.stride(-1) == 1 and k.stride(-1) == 1 and v.stride() == k.stride() and o.stride() == q.stride()
+    assert q.stride(2) == D and q.stride(1) == Hq * D
+    p = AttnParams()
+    p.q, p.k, p.v, p.o = _ptr(q), _ptr(k), _ptr(v), _ptr(o)
+    p.lse, p.mass = _ptr(lse), _ptr(mass)
+    p.n_layers, p.R, p.Hq, p.Hkv, p.D, p.n_ctx = L, R, Hq, Hkv, D, n_ctx
+    p.q_layer_stride = q.stride(0)
+    p.kv_layer_stride, p.kv_token_stride, p.kv_head_stride = k.stride(0), k.stride(1), k.stride(2)
+    p.mass_layer_stride = mass.stride(0) if (mass is not None and mass.dim() == 2) else T
+    p.softmax_scale = float(scale)
+    need = lib().pvlm_verify_attn_workspace_bytes(C.byref(p))
+    ws = workspace if workspace is not None else _workspace(q.device, "attn", need)
+    p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()
+    p._keep = (q, k, v, o, lse, mass, ws)
+    return p
+
+
+def verify_attn(q, k, v, n_ctx: int, *, want_lse: bool = True, want_mass: bool = False, scale: float = 0.0,
+                out=None, workspace=None):
+    """Window-verify GQA attention (see pvlm_verify_attn).  Returns (o, lse, mass)."""
+    _need_cuda(q, k, v)
+    batched = q.dim() == 4
+    L = q.shape[0] if batched else 1
+    R, Hq = q.shape[-3], q.shape[-2]
+    T = k.shape[-3]
+    o = out if out is not None else torch.empty_like(q)
+    lse = torch.empty((L, Hq, R) if batched else (Hq, R), dtype=torch.float32, device=q.device) if want_lse else None
+    mass = torch.empty((L, T) if batched else (T,), dtype=torch.float32, device=q.device) if want_mass else None
+    p = attn_params(q, k, v, n_ctx, o, lse, mass, scale, workspace)
+    st = lib().pvlm_verify_attn(C.byref(p), _stream(q.device))
+    if st != 0:
+        raise PvlmError(st, "pvlm_verify_attn")
+    return o, lse, mass
+
+
+def prune_params(mass_cur, mass_ref, vis_start, m, k, kept_idx, score, src_k, src_v, dst_k, dst_v,
+                 workspace=None) -> PruneParams:
+    p = PruneParams()
+    p.mass_cur, p.mass_ref = _ptr(mass_cur), _ptr(mass_ref)
+    p.vis_start, p.m, p.k = vis_start, m, k
+    p.kept_idx, p.score = _ptr(kept_idx), _ptr(score)
+    if src_k is not None:
+        if src_k.dim() == 3:
+            src_k, src_v, dst_k, dst_v = src_k[None], src_v[None], dst_k[None], dst_v[None]
+        L, S = src_k.shape[0], src_k.shape[1]
+        es = src_k.element_size()
+        row_bytes = src_k.shape[2] * src_k.shape[3] * es
+        assert src_k.stride(1) * es == row_bytes and dst_k.stride(1) * es == row_bytes, "rows must be dense"
+        assert src_v.stride() == src_k.stride() and dst_v.stride() == dst_k.stride()
+        p.src_k, p.src_v, p.dst_k, p.dst_v = _ptr(src_k), _ptr(src_v), _ptr(dst_k), _ptr(dst_v)
+        p.n_layers, p.src_len, p.row_bytes = L, S, row_bytes
+        p.src_layer_stride_bytes = src_k.stride(0) * es
+        p.dst_layer_stride_bytes = dst_k.stride(0) * es
+    need = lib().pvlm_uvprune_workspace_bytes(C.byref(p))
+    dev = mass_cur.device
+    ws = workspace if workspace is not None else _workspace(dev, "prune", need)
+    p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()
+    p._keep = (mass_cur, mass_ref, kept_idx, score, src_k, src_v, dst_k, dst_v, ws)
+    return p
+
+
+def uvprune_select_gather(mass_cur, mass_ref, vis_start: int, m: int, k: int, src_k=None, src_v=None, *,
+                          want_score: bool = False, workspace=None):
+    """UV-Prune select (+ gather if src_k/src_v given; see pvlm_uvprune_select_gather).
+
+    src_k/src_v: [L,S,Hkv,D] or [S,Hkv,D].  Returns (kept_idx int32 [k], score or None, dst_k, dst_v)."""
+    _need_cuda(mass_cur, mass_ref, src_k, src_v)
+    dev = mass_cur.device
+    kept = torch.empty(k, dtype=torch.int32, device=dev)
+    score = torch.empty(m, dtype=torch.float32, device=dev) if want_score else None
+    dst_k = dst_v = None
+    if src_k is not None:
+        shp = list(src_k.shape)
+        shp[-3] = shp[-3] - m + k
+        dst_k = torch.empty(shp, dtype=src_k.dtype, device=dev)
+        dst_v = torch.empty(shp, dtype=src_v.dtype, device=dev)
+    p = prune_params(mass_cur, mass_ref, vis_start, m, k, kept, score, src_k, src_v, dst_k, dst_v, workspace)
+    st = lib().pvlm_uvprune_select_gather(C.byref(p), _stream(dev))
+    if st != 0:
+        raise PvlmError(st, "pvlm_uvprune_select_gather")
+    return kept, score, dst_k, dst_v
+
+
+def accept_params(target_logits, draft_logits, draft_tokens, uniforms, temperature, outs: dict,
+                  workspace=None) -> AcceptParams:
+    tl, dl = target_logits, draft_logits
+    if tl.dim() == 2:
+        tl, dl = tl[None], dl[None]
+    B, R, V = tl.shape
+    gamma = R - 1
+    assert dl.shape == (B, gamma, V) and tl.dtype == torch.float32 and dl.dtype == torch.float32
+    assert tl.stride(2) == 1 and dl.stride(2) == 1
+    assert draft_tokens.dtype == torch.int32 and uniforms.dtype == torch.float32
+    assert draft_tokens.is_contiguous() and uniforms.is_contiguous()
+    p = AcceptParams()
+    p.target_logits, p.draft_logits = _ptr(tl), _ptr(dl)
+    p.target_row_stride, p.draft_row_stride = tl.stride(1), dl.stride(1)
+    p.target_batch_stride, p.draft_batch_stride = tl.stride(0), dl.stride(0)
+    p.draft_tokens, p.uniforms = _ptr(draft_tokens), _ptr(uniforms)
+    p.batch, p.gamma, p.V, p.temperature = B, gamma, V, float(temperature)
+    for name in ("n_accept", "out_tokens", "p_tok", "q_tok", "lse_p", "lse_q", "probs_p", "probs_q"):
+        setattr(p, name, _ptr(outs.get(name)))
+    need = lib().pvlm_spec_accept_workspace_bytes(C.byref(p))
+    ws = workspace if workspace is not None else _workspace(tl.device, "accept", need)
+    p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()
+    p._keep = (tl, dl, draft_tokens, uniforms, outs, ws)
+    return p
+
+
+def spec_accept(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0, *,
+                want_probs: bool = False, workspace=None) -> dict:
+    """Vocab softmax + accept/reject + residual resampling (see pvlm_spec_accept).
+
+    Shapes [gamma+1,V]/[gamma,V]/[gamma]/[gamma+1], or with a leading batch dimension."""
+    _need_cuda(target_logits, draft_logits, draft_tokens, uniforms)
+    dev = target_logits.device
+    batched = target_logits.dim() == 3
+    B = target_logits.shape[0] if batched else 1
+    gamma = target_logits.shape[-2] - 1
+    f32, i32 = torch.float32, torch.int32
+    outs = dict(n_accept=torch.empty(B, dtype=i32, device=dev),
+                out_tokens=torch.empty((B, gamma + 1), dtype=i32, device=dev),
+                p_tok=torch.empty((B, gamma), dtype=f32, device=dev),
+                q_tok=torch.empty((B, gamma), dtype=f32, device=dev),
+                lse_p=torch.empty((B, gamma + 1), dtype=f32, device=dev),
+                lse_q=torch.empty((B, gamma), dtype=f32, device=dev))
+    if want_probs:
+        outs["probs_p"] = torch.empty_like(target_logits)
+        outs["probs_q"] = torch.empty_like(draft_logits)
+    p = accept_params(target_logits, draft_logits, draft_tokens, uniforms, temperature, outs, workspace)
+    st = lib().pvlm_spec_accept(C.byref(p), _stream(dev))
+    if st != 0:
+        raise PvlmError(st, "pvlm_spec_accept")
+    if not batched:
+        outs = {k: (v[0] if k not in ("probs_p", "probs_q") else v) for k, v in outs.items()}
+    return outs

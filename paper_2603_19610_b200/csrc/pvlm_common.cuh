@@ -1,0 +1,53 @@
+// Shared host/device helpers of the pvlm library (internal).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "pvlm.h"
+
+namespace pvlm {
+
+constexpr int kNumSMs = 148;          // B200: 2 dies x 74 SMs
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+// Records a failed launch for pvlm_last_cuda_error(); returns PVLM_ERR_CUDA or PVLM_OK.
+pvlm_status check_launch();
+void set_cuda_error(int e);
+
+// ---- verify attention -----------------------------------------------------
+constexpr int kAttnBN = 64;           // keys per tile
+
+struct AttnPlan {
+  int rows;        // G * R valid rows per KV head
+  int n_warps;     // 16-row MMA tiles (one warp each)
+  int rows_pad;    // n_warps * 16
+  int T;           // keys per layer
+  int tiles;       // ceil(T / kAttnBN)
+  int splits;      // key-range splits per (layer, KV head)
+  int tiles_per_split;
+  size_t off_part_o, off_part_ml, off_lse2, off_part_mass, total;   // workspace layout (bytes)
+};
+bool make_attn_plan(const pvlm_attn_params& p, AttnPlan& plan);
+
+pvlm_status launch_verify_attn(const pvlm_attn_params& p, const AttnPlan& plan, cudaStream_t s);
+
+// ---- uvprune ----------------------------------------------------------------
+pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s);
+size_t uvprune_workspace(const pvlm_prune_params& p);
+
+// ---- accept -----------------------------------------------------------------
+struct AcceptPlan {
+  int rows;             // 2 * gamma + 1 logit rows per sequence
+  int stat_chunk, n_stat_chunks;      // row-statistics chunking over V
+  int samp_chunk, n_samp_chunks;      // resampling chunking over V
+  size_t off_stats, off_lse, off_n, off_csum, off_clast, total;
+};
+bool make_accept_plan(const pvlm_accept_params& p, AcceptPlan& plan);
+pvlm_status launch_spec_accept(const pvlm_accept_params& p, const AcceptPlan& plan, cudaStream_t s);
+
+}  // namespace pvlm

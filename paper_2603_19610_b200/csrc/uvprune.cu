@@ -1,0 +1,181 @@
+// UV-Prune: variation score, deterministic Top-K (radix select with
+// lower-index tie break, ascending output) and the row gather that builds the
+// compacted draft cache.
+#include "pvlm_common.cuh"
+
+namespace pvlm {
+
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+
+// Order-preserving map fp32 -> uint32 (larger float => larger key); -0.0 maps
+// with +0.0; NaN maps to 0 (below every number, -inf included).
+__device__ __forceinline__ uint32_t score_key(float s) {
+  if (s != s) return 0u;
+  uint32_t b = __float_as_uint(s + 0.0f);          // -0.0 + 0.0 = +0.0
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+struct SelArgs {
+  const float *cur, *ref;
+  float* score;
+  uint32_t* keys;     // workspace [m]
+  int* kept;
+  int m, k;
+};
+
+// Single CTA: m <= 2^24 elements, 4 radix passes of 8 bits over keys kept in
+// global/L2, then an ordered compaction.
+__global__ void __launch_bounds__(kSelThreads) uvprune_select_kernel(const SelArgs a) {
+  __shared__ unsigned int hist[256];
+  __shared__ unsigned int s_prefix, s_remaining;
+  __shared__ int warp_eq[kSelWarps], warp_sel[kSelWarps];
+  __shared__ int base_eq, base_sel;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // pass 0: scores and keys
+  for (int i = tid; i < a.m; i += kSelThreads) {
+    const float s = a.ref ? __fsub_rn(a.cur[i], a.ref[i]) : a.cur[i];
+    if (a.score) a.score[i] = s;
+    a.keys[i] = score_key(s);
+  }
+  if (tid == 0) { s_prefix = 0u; s_remaining = (unsigned)a.k; }
+  __syncthreads();
+  if (a.k == 0) return;
+
+  uint32_t mask = 0u;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (tid < 256) hist[tid] = 0u;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    for (int i0 = 0; i0 < a.m; i0 += kSelThreads) {      // uniform trip count: every lane reaches the ballot
+      const int i = i0 + tid;
+      const uint32_t key = (i < a.m) ? a.keys[i] : 0u;
+      const bool in = (i < a.m) && (key & mask) == prefix;
+      // warp-aggregated histogram update: lanes with the same digit elect one adder
+      const unsigned digit = (key >> shift) & 0xFFu;
+      const unsigned active = __ballot_sync(0xffffffffu, in);
+      if (in) {
+        const unsigned peers = __match_any_sync(active, digit);
+        if ((int)(__ffs(peers) - 1) == lane) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+      }
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned remaining = s_remaining, cum = 0u;
+      int d = 255;
+      for (; d > 0; --d) {
+        if (cum + hist[d] >= remaining) break;
+        cum += hist[d];
+      }
+      s_remaining = remaining - cum;           // how many to take from digit d's bucket
+      s_prefix = prefix | ((uint32_t)d << shift);
+    }
+    mask |= (0xFFu << shift);
+    __syncthreads();
+  }
+  const uint32_t tau = s_prefix;               // key of the k-th largest score
+  const int take_eq = (int)s_remaining;        // equals to keep, lowest indices first
+
+  if (tid == 0) { base_eq = 0; base_sel = 0; }
+  __syncthreads();
+  for (int i0 = 0; i0 < a.m; i0 += kSelThreads) {
+    const int i = i0 + tid;
+    const uint32_t key = (i < a.m) ? a.keys[i] : 0u;
+    const bool gt = (i < a.m) && key > tau;
+    const bool eq = (i < a.m) && key == tau;
+    const unsigned eq_b = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) warp_eq[warp] = __popc(eq_b);
+    __syncthreads();
+    int eq_before = base_eq + __popc(eq_b & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) eq_before += warp_eq[w];
+    const bool sel = gt || (eq && eq_before < take_eq);
+    const unsigned sel_b = __ballot_sync(0xffffffffu, sel);
+    if (lane == 0) warp_sel[warp] = __popc(sel_b);
+    __syncthreads();
+    int pos = base_sel + __popc(sel_b & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) pos += warp_sel[w];
+    if (sel) a.kept[pos] = i;
+    __syncthreads();
+    if (tid == kSelThreads - 1) {
+      base_eq = eq_before + (eq ? 1 : 0);
+      base_sel = pos + (sel ? 1 : 0);
+    }
+    __syncthreads();
+  }
+}
+
+struct GatherArgs {
+  const int4 *src_k, *src_v;
+  int4 *dst_k, *dst_v;
+  const int* kept;
+  int vis_start, m, k, dst_len, n_layers;
+  int row_vec;                       // 16-byte units per row
+  long long src_ls_vec, dst_ls_vec;  // layer strides in 16-byte units
+};
+
+// One thread moves 16 bytes of K and 16 bytes of V per step; a destination row
+// maps to its source row through the kept-index list.
+__global__ void __launch_bounds__(256) uvprune_gather_kernel(const GatherArgs a) {
+  const long long per_layer = (long long)a.dst_len * a.row_vec;
+  const long long total = per_layer * a.n_layers;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += stride) {
+    const int layer = (int)(u / per_layer);
+    const long long w = u - (long long)layer * per_layer;
+    const int drow = (int)(w / a.row_vec);
+    const int c = (int)(w - (long long)drow * a.row_vec);
+    int srow;
+    if (drow < a.vis_start) srow = drow;
+    else if (drow < a.vis_start + a.k) srow = a.vis_start + __ldg(a.kept + (drow - a.vis_start));
+    else srow = drow - a.k + a.m;
+    const long long so = (long long)layer * a.src_ls_vec + (long long)srow * a.row_vec + c;
+    const long long dof = (long long)layer * a.dst_ls_vec + (long long)drow * a.row_vec + c;
+    const int4 kk = __ldg(a.src_k + so);
+    const int4 vv = __ldg(a.src_v + so);
+    a.dst_k[dof] = kk;
+    a.dst_v[dof] = vv;
+  }
+}
+
+}  // namespace
+
+size_t uvprune_workspace(const pvlm_prune_params& p) { return align_up((size_t)(p.m > 0 ? p.m : 1) * 4, 256); }
+
+pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s) {
+  SelArgs sa;
+  sa.cur = p.mass_cur + p.vis_start;
+  sa.ref = p.mass_ref ? p.mass_ref + p.vis_start : nullptr;
+  sa.score = p.score;
+  sa.keys = (uint32_t*)p.workspace;
+  sa.kept = p.kept_idx;
+  sa.m = p.m;
+  sa.k = p.k;
+  if (p.m > 0) uvprune_select_kernel<<<1, kSelThreads, 0, s>>>(sa);
+  if (p.src_k) {
+    GatherArgs g;
+    g.src_k = (const int4*)p.src_k;
+    g.src_v = (const int4*)p.src_v;
+    g.dst_k = (int4*)p.dst_k;
+    g.dst_v = (int4*)p.dst_v;
+    g.kept = p.kept_idx;
+    g.vis_start = p.vis_start; g.m = p.m; g.k = p.k;
+    g.dst_len = p.src_len - p.m + p.k;
+    g.n_layers = p.n_layers;
+    g.row_vec = (int)(p.row_bytes / 16);
+    g.src_ls_vec = p.src_layer_stride_bytes / 16;
+    g.dst_ls_vec = p.dst_layer_stride_bytes / 16;
+    const long long total = (long long)g.dst_len * g.row_vec * g.n_layers;
+    if (total > 0) {
+      long long blocks = (total + 255) / 256;
+      const long long cap = (long long)kNumSMs * 16;
+      if (blocks > cap) blocks = cap;
+      uvprune_gather_kernel<<<(int)blocks, 256, 0, s>>>(g);
+    }
+  }
+  return check_launch();
+}
+
+}  // namespace pvlm

@@ -1,0 +1,96 @@
+"""The C-ABI library loads without a GPU, exports every symbol the header
+declares, the header is valid C99, and the ctypes mirrors match its layout."""
+import ctypes as C
+import os
+import re
+import subprocess
+import sys
+import tempfile
+
+import pytest
+
+from paper_2603_19610_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "pvlm.h")
+
+
+def declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(pvlm_[a-z_0-9]+)\s*\(", src)))
+
+
+def test_exports_every_declared_symbol():
+    L = binding.lib()
+    names = declared_functions()
+    assert len(names) >= 9
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(binding.EXPORTS) <= set(names)
+    assert L.pvlm_version() >= 1000
+    assert L.pvlm_status_string(0) == b"PVLM_OK"
+    assert L.pvlm_status_string(3) == b"PVLM_ERR_WORKSPACE"
+
+
+def test_header_is_c99_and_layouts_match():
+    fields = {"pvlm_attn_params": binding.AttnParams, "pvlm_prune_params": binding.PruneParams,
+              "pvlm_accept_params": binding.AcceptParams}
+    prog = ['#include <stdio.h>', '#include <stddef.h>', '#include "pvlm.h"', 'int main(void){']
+    for cname, st in fields.items():
+        prog.append(f'printf("{cname} %zu\\n", sizeof({cname}));')
+        for fname, _ in st._fields_:
+            prog.append(f'printf("{cname}.{fname} %zu\\n", offsetof({cname}, {fname}));')
+    prog.append("return 0;}")
+    with tempfile.TemporaryDirectory() as td:
+        src = os.path.join(td, "layout.c")
+        open(src, "w").write("\n".join(prog))
+        exe = os.path.join(td, "layout")
+        subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
+                        src, "-o", exe], check=True)
+        out = subprocess.run([exe], check=True, capture_output=True, text=True).stdout
+    got = dict(line.split() for line in out.strip().splitlines())
+    for cname, st in fields.items():
+        assert int(got[cname]) == C.sizeof(st)
+        for fname, _ in st._fields_:
+            assert int(got[f"{cname}.{fname}"]) == getattr(st, fname).offset, (cname, fname)
+
+
+def test_workspace_queries_and_argument_errors_need_no_gpu():
+    L = binding.lib()
+    p = binding.AttnParams()
+    p.n_layers, p.R, p.Hq, p.Hkv, p.D, p.n_ctx = 64, 13, 40, 8, 128, 32768
+    ws = L.pvlm_verify_attn_workspace_bytes(C.byref(p))
+    assert 0 < ws < (1 << 30)
+    p.D = 96
+    assert L.pvlm_verify_attn_workspace_bytes(C.byref(p)) == 0
+    assert L.pvlm_verify_attn(C.byref(p), None) == 1                    # NULL tensors: invalid before any launch
+    p.q = p.k = p.v = p.o = 4096
+    assert L.pvlm_verify_attn(C.byref(p), None) == 2                    # D = 96 unsupported
+    p.D = 128
+    p.kv_head_stride, p.kv_token_stride = 128, 8 * 128
+    p.kv_layer_stride, p.q_layer_stride = 32781 * 1024, 13 * 40 * 128
+    assert L.pvlm_verify_attn(C.byref(p), None) == 3                    # no workspace
+    p.Hq = 41
+    assert L.pvlm_verify_attn(C.byref(p), None) == 2                    # Hq % Hkv != 0
+
+    a = binding.AcceptParams()
+    a.batch, a.gamma, a.V = 1, 12, 152064
+    assert L.pvlm_spec_accept_workspace_bytes(C.byref(a)) > 0
+    assert L.pvlm_spec_accept(C.byref(a), None) == 1
+    a.gamma = 65
+    assert L.pvlm_spec_accept_workspace_bytes(C.byref(a)) == 0
+
+    u = binding.PruneParams()
+    u.m, u.k = 100, 101
+    assert L.pvlm_uvprune_select_gather(C.byref(u), None) == 1          # k > m
+    u.k = 10
+    assert L.pvlm_uvprune_workspace_bytes(C.byref(u)) >= 400
+    assert L.pvlm_uvprune_select_gather(C.byref(u), None) == 1          # no mass pointer
+
+
+def test_no_cpu_fallback():
+    import torch
+    q = torch.zeros(2, 4, 64, dtype=torch.bfloat16)
+    with pytest.raises(RuntimeError):
+        binding.verify_attn(q, torch.zeros(10, 1, 64, dtype=torch.bfloat16), torch.zeros(10, 1, 64, dtype=torch.bfloat16), 8)
