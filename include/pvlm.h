@@ -75,8 +75,14 @@ typedef struct {
   const void *v;        /* bf16, same layout and strides as k                                  */
   void *o;              /* bf16 [n_layers][R][Hq][D], same layer stride as q                   */
   float *lse;           /* fp32 [n_layers][Hq][R] natural-log lse; nullable                    */
-  float *mass;          /* fp32 [n_layers][T], layer stride mass_layer_stride; nullable =>
-                           the mass pass is skipped for the whole call                         */
+  float *mass;          /* fp32 [n_mass][T], row stride mass_layer_stride; nullable => the
+                           mass pass is skipped for the whole call.  n_mass = n_mass_layers
+                           if mass_layers is given, else n_layers                              */
+  const int *mass_layers; /* HOST array [n_mass_layers] of layer indices (each in
+                           [0, n_layers)) whose mass is wanted, row i of `mass` receiving
+                           layer mass_layers[i]; NULL => every layer.  At most 8 entries.
+                           The variation score needs only its two end layers (Eq. 2).          */
+  int n_mass_layers;
   int n_layers, R, Hq, Hkv, D, n_ctx;
   long long q_layer_stride;    /* elements */
   long long kv_layer_stride;   /* elements */
@@ -171,6 +177,46 @@ typedef struct {
 
 size_t pvlm_spec_accept_workspace_bytes(const pvlm_accept_params *p);
 pvlm_status pvlm_spec_accept(const pvlm_accept_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
+ * One whole verify -> prune -> accept step from HOST-side step inputs.
+ *
+ * The verification round of the parallel decoding pipeline (paper Sec. 4.2,
+ * Stage II; Appendix B) as one call: copy this step's inputs from host memory
+ * into caller-provided device buffers, run the three stages in order on
+ * `stream`, copy the step's results back.  The KV cache of the committed
+ * context is resident device state (like weights) and is not copied; only the
+ * window's own K/V rows are written into it at token rows [n_ctx, n_ctx + R).
+ *
+ * `attn`, `prune`, `accept` are complete parameter blocks as for the three
+ * calls above (all their pointers are device pointers; prune.mass_cur /
+ * mass_ref normally point at rows of attn.mass).  A stage whose `run_*` flag
+ * is 0 is skipped.  Every h_* pointer is a HOST pointer (pinned memory makes
+ * the copies asynchronous) and may be NULL, which skips that copy:
+ *   h_q            bf16 [n_layers][R][Hq][D]        -> attn.q
+ *   h_k_window/v   bf16 [n_layers][R][Hkv][D]       -> attn.k / attn.v rows n_ctx.. (needs
+ *                                                      kv_head_stride == D, kv_token_stride == Hkv*D)
+ *   h_target_logits fp32 [batch][gamma+1][V] dense  -> accept.target_logits (dense strides required)
+ *   h_draft_logits  fp32 [batch][gamma][V] dense    -> accept.draft_logits
+ *   h_draft_tokens, h_uniforms                      -> accept.draft_tokens, accept.uniforms
+ *   h_o            <- attn.o;  h_n_accept, h_out_tokens <- accept;  h_kept_idx <- prune.kept_idx
+ * The call returns after enqueueing; results in host memory are valid once
+ * the stream has been synchronised by the caller.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+  pvlm_attn_params attn;
+  pvlm_prune_params prune;
+  pvlm_accept_params accept;
+  int run_attn, run_prune, run_accept;
+  const void *h_q, *h_k_window, *h_v_window;
+  const float *h_target_logits, *h_draft_logits;
+  const int *h_draft_tokens;
+  const float *h_uniforms;
+  void *h_o;
+  int *h_n_accept, *h_out_tokens, *h_kept_idx;
+} pvlm_step_params;
+
+pvlm_status pvlm_verify_step(const pvlm_step_params *p, void *stream);
 
 #ifdef __cplusplus
 }

@@ -31,6 +31,7 @@ class PvlmError(RuntimeError):
 class AttnParams(C.Structure):
     _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("o", C.c_void_p),
                 ("lse", C.c_void_p), ("mass", C.c_void_p),
+                ("mass_layers", C.POINTER(C.c_int)), ("n_mass_layers", C.c_int),
                 ("n_layers", C.c_int), ("R", C.c_int), ("Hq", C.c_int), ("Hkv", C.c_int), ("D", C.c_int),
                 ("n_ctx", C.c_int),
                 ("q_layer_stride", C.c_longlong), ("kv_layer_stride", C.c_longlong),
@@ -63,10 +64,20 @@ class AcceptParams(C.Structure):
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
+class StepParams(C.Structure):
+    _fields_ = [("attn", AttnParams), ("prune", PruneParams), ("accept", AcceptParams),
+                ("run_attn", C.c_int), ("run_prune", C.c_int), ("run_accept", C.c_int),
+                ("h_q", C.c_void_p), ("h_k_window", C.c_void_p), ("h_v_window", C.c_void_p),
+                ("h_target_logits", C.c_void_p), ("h_draft_logits", C.c_void_p),
+                ("h_draft_tokens", C.c_void_p), ("h_uniforms", C.c_void_p),
+                ("h_o", C.c_void_p), ("h_n_accept", C.c_void_p), ("h_out_tokens", C.c_void_p),
+                ("h_kept_idx", C.c_void_p)]
+
+
 EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
            "pvlm_verify_attn_workspace_bytes", "pvlm_verify_attn",
            "pvlm_uvprune_workspace_bytes", "pvlm_uvprune_select_gather",
-           "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept")
+           "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept", "pvlm_verify_step")
 
 
 def lib() -> C.CDLL:
@@ -85,7 +96,7 @@ def lib() -> C.CDLL:
                 f.restype = C.c_size_t
                 f.argtypes = [C.POINTER(st)]
             for name, st in (("pvlm_verify_attn", AttnParams), ("pvlm_uvprune_select_gather", PruneParams),
-                             ("pvlm_spec_accept", AcceptParams)):
+                             ("pvlm_spec_accept", AcceptParams), ("pvlm_verify_step", StepParams)):
                 f = getattr(L, name)
                 f.restype = C.c_int
                 f.argtypes = [C.POINTER(st), C.c_void_p]
@@ -120,7 +131,7 @@ def _stream(dev):
     return C.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
 
 
-def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None) -> AttnParams:
+def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None, mass_layers=None) -> AttnParams:
     """Fill an AttnParams from torch tensors: q/o [L,R,Hq,D] or [R,Hq,D]; k/v [L,T,Hkv,D] or [T,Hkv,D]."""
     if q.dim() == 3:
         q, k, v, o = q[None], k[None], v[None], o[None]
@@ -133,6 +144,10 @@ def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None) -> Attn
     p = AttnParams()
     p.q, p.k, p.v, p.o = _ptr(q), _ptr(k), _ptr(v), _ptr(o)
     p.lse, p.mass = _ptr(lse), _ptr(mass)
+    ml = None
+    if mass is not None and mass_layers is not None:
+        ml = (C.c_int * len(mass_layers))(*[int(x) for x in mass_layers])
+        p.mass_layers, p.n_mass_layers = ml, len(mass_layers)
     p.n_layers, p.R, p.Hq, p.Hkv, p.D, p.n_ctx = L, R, Hq, Hkv, D, n_ctx
     p.q_layer_stride = q.stride(0)
     p.kv_layer_stride, p.kv_token_stride, p.kv_head_stride = k.stride(0), k.stride(1), k.stride(2)
@@ -141,13 +156,16 @@ def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None) -> Attn
     need = lib().pvlm_verify_attn_workspace_bytes(C.byref(p))
     ws = workspace if workspace is not None else _workspace(q.device, "attn", need)
     p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()
-    p._keep = (q, k, v, o, lse, mass, ws)
+    p._keep = (q, k, v, o, lse, mass, ws, ml)
     return p
 
 
 def verify_attn(q, k, v, n_ctx: int, *, want_lse: bool = True, want_mass: bool = False, scale: float = 0.0,
-                out=None, workspace=None):
-    """Window-verify GQA attention (see pvlm_verify_attn).  Returns (o, lse, mass)."""
+                out=None, workspace=None, mass_layers=None):
+    """Window-verify GQA attention (see pvlm_verify_attn).  Returns (o, lse, mass).
+
+    mass_layers (batched form only): list of layer indices whose mass is wanted;
+    mass then has one row per listed layer."""
     _need_cuda(q, k, v)
     batched = q.dim() == 4
     L = q.shape[0] if batched else 1
@@ -155,8 +173,9 @@ def verify_attn(q, k, v, n_ctx: int, *, want_lse: bool = True, want_mass: bool =
     T = k.shape[-3]
     o = out if out is not None else torch.empty_like(q)
     lse = torch.empty((L, Hq, R) if batched else (Hq, R), dtype=torch.float32, device=q.device) if want_lse else None
-    mass = torch.empty((L, T) if batched else (T,), dtype=torch.float32, device=q.device) if want_mass else None
-    p = attn_params(q, k, v, n_ctx, o, lse, mass, scale, workspace)
+    n_mass = len(mass_layers) if mass_layers is not None else L
+    mass = torch.empty((n_mass, T) if batched else (T,), dtype=torch.float32, device=q.device) if want_mass else None
+    p = attn_params(q, k, v, n_ctx, o, lse, mass, scale, workspace, mass_layers if want_mass else None)
     st = lib().pvlm_verify_attn(C.byref(p), _stream(q.device))
     if st != 0:
         raise PvlmError(st, "pvlm_verify_attn")
@@ -264,3 +283,33 @@ def spec_accept(target_logits, draft_logits, draft_tokens, uniforms, temperature
     if not batched:
         outs = {k: (v[0] if k not in ("probs_p", "probs_q") else v) for k, v in outs.items()}
     return outs
+
+
+def verify_step(attn: AttnParams | None, prune: PruneParams | None, accept: AcceptParams | None, *,
+                host_in: dict | None = None, host_out: dict | None = None, device=None) -> StepParams:
+    """One whole verify -> prune -> accept step through pvlm_verify_step.
+
+    attn / prune / accept are parameter blocks built by attn_params / prune_params /
+    accept_params (None skips the stage).  host_in maps h_q, h_k_window, h_v_window,
+    h_target_logits, h_draft_logits, h_draft_tokens, h_uniforms to (pinned) CPU tensors
+    copied to the device first; host_out maps h_o, h_n_accept, h_out_tokens, h_kept_idx to
+    CPU tensors filled at the end.  Asynchronous: synchronise the stream before reading."""
+    sp = StepParams()
+    keep = []
+    for name, blk in (("attn", attn), ("prune", prune), ("accept", accept)):
+        if blk is not None:
+            setattr(sp, name, blk)
+            setattr(sp, "run_" + name, 1)
+            keep.append(blk)
+    for d in (host_in, host_out):
+        for k, t in (d or {}).items():
+            if t is not None:
+                assert not t.is_cuda and t.is_contiguous()
+                setattr(sp, k, C.c_void_p(t.data_ptr()))
+                keep.append(t)
+    dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+    st = lib().pvlm_verify_step(C.byref(sp), _stream(dev))
+    if st != 0:
+        raise PvlmError(st, "pvlm_verify_step")
+    sp._keep = keep
+    return sp

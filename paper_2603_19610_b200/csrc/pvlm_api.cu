@@ -63,7 +63,16 @@ pvlm_status pvlm_verify_attn(const pvlm_attn_params* p, void* stream) {
   if (p->n_layers > 1) {
     if (p->kv_layer_stride < (long long)plan.T * p->kv_token_stride || p->kv_layer_stride % 8) return PVLM_ERR_INVALID_ARG;
     if (p->q_layer_stride < (long long)p->R * p->Hq * p->D || p->q_layer_stride % 8) return PVLM_ERR_INVALID_ARG;
-    if (p->mass && p->mass_layer_stride < plan.T) return PVLM_ERR_INVALID_ARG;
+  }
+  if (p->mass) {
+    const int n_mass = p->mass_layers ? p->n_mass_layers : p->n_layers;
+    if (p->mass_layers) {
+      if (p->n_mass_layers < 1) return PVLM_ERR_INVALID_ARG;
+      if (p->n_mass_layers > 8) return PVLM_ERR_UNSUPPORTED;
+      for (int i = 0; i < p->n_mass_layers; ++i)
+        if (p->mass_layers[i] < 0 || p->mass_layers[i] >= p->n_layers) return PVLM_ERR_INVALID_ARG;
+    }
+    if (n_mass > 1 && p->mass_layer_stride < plan.T) return PVLM_ERR_INVALID_ARG;
   }
   if (p->n_layers > 65535 || p->Hkv > 65535) return PVLM_ERR_UNSUPPORTED;
   const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, plan.total);
@@ -125,6 +134,71 @@ pvlm_status pvlm_spec_accept(const pvlm_accept_params* p, void* stream) {
   const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, plan.total);
   if (w != PVLM_OK) return w;
   return launch_spec_accept(*p, plan, (cudaStream_t)stream);
+}
+
+pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
+  if (!p) return PVLM_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const pvlm_attn_params& a = p->attn;
+  const pvlm_accept_params& c = p->accept;
+  cudaError_t e = cudaSuccess;
+  auto ok = [&]() { return e == cudaSuccess; };
+  // ---- host -> device: this step's inputs ----
+  if (p->run_attn) {
+    if (a.n_layers < 1 || a.R < 1 || a.Hq < 1 || a.Hkv < 1 || a.D < 1 || a.n_ctx < 0) return PVLM_ERR_INVALID_ARG;
+    const size_t q_layer = (size_t)a.R * a.Hq * a.D * 2;
+    if (p->h_q && ok())
+      e = cudaMemcpy2DAsync(const_cast<void*>(a.q), (size_t)a.q_layer_stride * 2, p->h_q, q_layer, q_layer, a.n_layers,
+                            cudaMemcpyHostToDevice, s);
+    if (p->h_k_window || p->h_v_window) {
+      if (a.kv_head_stride != a.D || a.kv_token_stride != (long long)a.Hkv * a.D) return PVLM_ERR_UNSUPPORTED;
+      const size_t w_layer = (size_t)a.R * a.Hkv * a.D * 2;
+      const size_t row0 = (size_t)a.n_ctx * a.kv_token_stride * 2;
+      const size_t pitch = a.n_layers > 1 ? (size_t)a.kv_layer_stride * 2 : w_layer;
+      if (p->h_k_window && ok())
+        e = cudaMemcpy2DAsync((char*)const_cast<void*>(a.k) + row0, pitch, p->h_k_window, w_layer, w_layer, a.n_layers,
+                              cudaMemcpyHostToDevice, s);
+      if (p->h_v_window && ok())
+        e = cudaMemcpy2DAsync((char*)const_cast<void*>(a.v) + row0, pitch, p->h_v_window, w_layer, w_layer, a.n_layers,
+                              cudaMemcpyHostToDevice, s);
+    }
+  }
+  if (p->run_accept) {
+    if (c.gamma < 1 || c.V < 1 || c.batch < 1) return PVLM_ERR_INVALID_ARG;
+    if (p->h_target_logits || p->h_draft_logits) {
+      if (c.target_row_stride != c.V || c.draft_row_stride != c.V) return PVLM_ERR_UNSUPPORTED;
+      if (c.batch > 1 && (c.target_batch_stride != (long long)(c.gamma + 1) * c.V ||
+                          c.draft_batch_stride != (long long)c.gamma * c.V)) return PVLM_ERR_UNSUPPORTED;
+    }
+    const size_t B = (size_t)c.batch;
+    if (p->h_target_logits && ok())
+      e = cudaMemcpyAsync(const_cast<float*>(c.target_logits), p->h_target_logits, B * (c.gamma + 1) * c.V * 4, cudaMemcpyHostToDevice, s);
+    if (p->h_draft_logits && ok())
+      e = cudaMemcpyAsync(const_cast<float*>(c.draft_logits), p->h_draft_logits, B * c.gamma * c.V * 4, cudaMemcpyHostToDevice, s);
+    if (p->h_draft_tokens && ok())
+      e = cudaMemcpyAsync(const_cast<int*>(c.draft_tokens), p->h_draft_tokens, B * c.gamma * 4, cudaMemcpyHostToDevice, s);
+    if (p->h_uniforms && ok())
+      e = cudaMemcpyAsync(const_cast<float*>(c.uniforms), p->h_uniforms, B * (c.gamma + 1) * 4, cudaMemcpyHostToDevice, s);
+  }
+  if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+  // ---- the three stages ----
+  pvlm_status st;
+  if (p->run_attn && (st = pvlm_verify_attn(&p->attn, stream)) != PVLM_OK) return st;
+  if (p->run_prune && (st = pvlm_uvprune_select_gather(&p->prune, stream)) != PVLM_OK) return st;
+  if (p->run_accept && (st = pvlm_spec_accept(&p->accept, stream)) != PVLM_OK) return st;
+  // ---- device -> host: this step's results ----
+  if (p->run_attn && p->h_o) {
+    const size_t q_layer = (size_t)a.R * a.Hq * a.D * 2;
+    e = cudaMemcpy2DAsync(p->h_o, q_layer, a.o, (size_t)a.q_layer_stride * 2, q_layer, a.n_layers, cudaMemcpyDeviceToHost, s);
+  }
+  if (p->run_prune && p->h_kept_idx && p->prune.k > 0 && ok())
+    e = cudaMemcpyAsync(p->h_kept_idx, p->prune.kept_idx, (size_t)p->prune.k * 4, cudaMemcpyDeviceToHost, s);
+  if (p->run_accept && p->h_n_accept && ok())
+    e = cudaMemcpyAsync(p->h_n_accept, c.n_accept, (size_t)c.batch * 4, cudaMemcpyDeviceToHost, s);
+  if (p->run_accept && p->h_out_tokens && ok())
+    e = cudaMemcpyAsync(p->h_out_tokens, c.out_tokens, (size_t)c.batch * (c.gamma + 1) * 4, cudaMemcpyDeviceToHost, s);
+  if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+  return PVLM_OK;
 }
 
 }  // extern "C"

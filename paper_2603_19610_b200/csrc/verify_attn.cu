@@ -22,6 +22,9 @@ struct AttnArgs {
   int R, Hq, Hkv, G, n_ctx, T, T_pad, rows, rows_pad, splits, tiles_per_split, tiles;
   long long q_ls, kv_ls, kv_ts, kv_hs, mass_ls;
   float scale_log2;
+  int n_mass;            // mass rows to produce
+  int mass_layer[8];     // layer of mass row i (when listed; identity otherwise)
+  int mass_listed;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -65,8 +68,10 @@ constexpr int kStages = 3;
 
 // MODE 0: online-softmax attention over the CTA's key range (partials or final O).
 // MODE 1: mass pass: P = exp2(s - lse2) summed over the group's rows per key.
-template <int D, int MODE>
-__global__ void __launch_bounds__(256) attn_kernel(const AttnArgs a) {
+// MAXW = most warps a CTA may have: up to 6 warps the register budget is held to 168 so that
+// two CTAs (3 warps per scheduler) stay resident per SM.
+template <int D, int MODE, int MAXW>
+__global__ void __launch_bounds__(MAXW * 32, MAXW <= 6 ? 2 : 1) attn_kernel(const AttnArgs a) {
   constexpr int BN = kAttnBN;
   constexpr int CHUNKS = D / 8;
   constexpr int ROW_BYTES = D * 2;
@@ -76,7 +81,9 @@ __global__ void __launch_bounds__(256) attn_kernel(const AttnArgs a) {
   const uint32_t smem_base = smem_u32(smem);
   float* colsum = reinterpret_cast<float*>(smem + kStages * STAGE_BYTES);   // MODE 1 only: [8][BN]
 
-  const int split = blockIdx.x, kvh = blockIdx.y, layer = blockIdx.z;
+  const int split = blockIdx.x, kvh = blockIdx.y;
+  const int zrow = blockIdx.z;            // MODE 0: the layer; MODE 1: the mass row
+  const int layer = (MODE == 1 && a.mass_listed) ? a.mass_layer[zrow] : zrow;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile_begin = split * a.tiles_per_split;
   const int n_tiles = min(a.tiles, tile_begin + a.tiles_per_split) - tile_begin;
@@ -252,7 +259,7 @@ __global__ void __launch_bounds__(256) attn_kernel(const AttnArgs a) {
         float acc = 0.f;
         const int nw = blockDim.x >> 5;
         for (int w = 0; w < nw; ++w) acc += colsum[w * BN + t];
-        a.part_mass[((long long)layer * a.Hkv + kvh) * a.T_pad + j0 + t] = acc;
+        a.part_mass[((long long)zrow * a.Hkv + kvh) * a.T_pad + j0 + t] = acc;
       }
     }
   }
@@ -343,21 +350,28 @@ __global__ void mass_reduce_kernel(const AttnArgs a) {
   a.mass[(long long)layer * a.mass_ls + j] = acc;
 }
 
-template <int D>
-pvlm_status launch_d(const AttnArgs& a, const pvlm_attn_params& p, const AttnPlan& plan, cudaStream_t s) {
+template <int D, int MAXW>
+pvlm_status launch_dw(const AttnArgs& a, const pvlm_attn_params& p, const AttnPlan& plan, cudaStream_t s) {
   const dim3 grid(plan.splits, p.Hkv, p.n_layers);
   const int threads = plan.n_warps * 32;
   const int smem0 = kStages * 2 * kAttnBN * D * 2;
-  cudaFuncSetAttribute(attn_kernel<D, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0);
-  attn_kernel<D, 0><<<grid, threads, smem0, s>>>(a);
+  cudaFuncSetAttribute(attn_kernel<D, 0, MAXW>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0);
+  cudaFuncSetAttribute(attn_kernel<D, 0, MAXW>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+  attn_kernel<D, 0, MAXW><<<grid, threads, smem0, s>>>(a);
   if (plan.splits > 1) attn_combine_kernel<D><<<dim3(plan.rows, p.Hkv, p.n_layers), D, 0, s>>>(a);
   if (p.mass) {
     const int smem1 = kStages * kAttnBN * D * 2 + 8 * kAttnBN * 4;
-    cudaFuncSetAttribute(attn_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1);
-    attn_kernel<D, 1><<<grid, threads, smem1, s>>>(a);
-    mass_reduce_kernel<<<dim3(ceil_div(plan.T, 256), p.n_layers), 256, 0, s>>>(a);
+    cudaFuncSetAttribute(attn_kernel<D, 1, MAXW>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1);
+    cudaFuncSetAttribute(attn_kernel<D, 1, MAXW>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+    attn_kernel<D, 1, MAXW><<<dim3(plan.splits, p.Hkv, a.n_mass), threads, smem1, s>>>(a);
+    mass_reduce_kernel<<<dim3(ceil_div(plan.T, 256), a.n_mass), 256, 0, s>>>(a);
   }
   return check_launch();
+}
+
+template <int D>
+pvlm_status launch_d(const AttnArgs& a, const pvlm_attn_params& p, const AttnPlan& plan, cudaStream_t s) {
+  return plan.n_warps <= 6 ? launch_dw<D, 6>(a, p, plan, s) : launch_dw<D, 8>(a, p, plan, s);
 }
 
 }  // namespace
@@ -386,7 +400,10 @@ bool make_attn_plan(const pvlm_attn_params& p, AttnPlan& plan) {
   plan.off_lse2 = off;
   off += align_up((size_t)p.n_layers * p.Hq * p.R * 4, 256);
   plan.off_part_mass = off;
-  if (p.mass) off += align_up((size_t)items * align_up(plan.T, kAttnBN) * 4, 256);
+  if (p.mass) {
+    const int n_mass = p.mass_layers ? p.n_mass_layers : p.n_layers;
+    off += align_up((size_t)n_mass * p.Hkv * align_up(plan.T, kAttnBN) * 4, 256);
+  }
   plan.total = off;
   return true;
 }
@@ -412,6 +429,9 @@ pvlm_status launch_verify_attn(const pvlm_attn_params& p, const AttnPlan& plan, 
   a.mass_ls = p.mass_layer_stride;
   const float scale = (p.softmax_scale == 0.f) ? 1.0f / sqrtf((float)p.D) : p.softmax_scale;
   a.scale_log2 = scale * kLog2e;
+  a.mass_listed = p.mass_layers != nullptr;
+  a.n_mass = a.mass_listed ? p.n_mass_layers : p.n_layers;
+  for (int i = 0; i < 8; ++i) a.mass_layer[i] = (a.mass_listed && i < p.n_mass_layers) ? p.mass_layers[i] : 0;
   return p.D == 64 ? launch_d<64>(a, p, plan, s) : launch_d<128>(a, p, plan, s);
 }
 

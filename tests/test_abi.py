@@ -24,7 +24,7 @@ def declared_functions():
 def test_exports_every_declared_symbol():
     L = binding.lib()
     names = declared_functions()
-    assert len(names) >= 9
+    assert len(names) >= 10
     for n in names:
         assert hasattr(L, n), n
     assert set(binding.EXPORTS) <= set(names)
@@ -35,7 +35,7 @@ def test_exports_every_declared_symbol():
 
 def test_header_is_c99_and_layouts_match():
     fields = {"pvlm_attn_params": binding.AttnParams, "pvlm_prune_params": binding.PruneParams,
-              "pvlm_accept_params": binding.AcceptParams}
+              "pvlm_accept_params": binding.AcceptParams, "pvlm_step_params": binding.StepParams}
     prog = ['#include <stdio.h>', '#include <stddef.h>', '#include "pvlm.h"', 'int main(void){']
     for cname, st in fields.items():
         prog.append(f'printf("{cname} %zu\\n", sizeof({cname}));')

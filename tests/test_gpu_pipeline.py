@@ -1,0 +1,152 @@
+"""End to end: verify attention -> mass -> UV-Prune -> gather -> accept on the five
+workload configurations, GPU against oracle, with the tolerance bands for decisions that
+floating point can flip; the whole-step C-ABI entry with host buffers; two streams."""
+import numpy as np
+import pytest
+import torch
+
+from oracle.accept import spec_accept as oracle_accept
+from oracle.attention import verify_attn as oracle_attn
+from oracle.uvprune import gather_rows, score_fp32, select_topk
+from paper_2603_19610_b200 import binding, workloads as wl
+from helpers import assert_o_close, assert_rel_close, bf16_cuda, bits_of
+
+pytestmark = pytest.mark.gpu
+
+
+def layers_for(cfg):
+    """(reference layer inputs, current layer inputs) of a config."""
+    if cfg.n_layers > 1:
+        return wl.attn_layer(cfg, cfg.ref_layer), wl.attn_layer(cfg, cfg.cur_layer)
+    return wl.attn_layer(cfg, 0, role="ref"), wl.attn_layer(cfg, 0)
+
+
+@pytest.mark.parametrize("cid", [0, 1, 2, 3, 4])
+def test_config_end_to_end(cid):
+    cfg = wl.CONFIGS[cid]
+    ref_in, cur_in = layers_for(cfg)
+    # ---- GPU: both mass layers in one batched launch, then prune (2-layer cache), then accept
+    q = torch.stack([bf16_cuda(ref_in[0]), bf16_cuda(cur_in[0])])
+    k = torch.stack([bf16_cuda(ref_in[1]), bf16_cuda(cur_in[1])])
+    v = torch.stack([bf16_cuda(ref_in[2]), bf16_cuda(cur_in[2])])
+    o, lse, mass = binding.verify_attn(q, k, v, cfg.n_ctx, want_mass=True, mass_layers=[0, 1])
+    kept, score, dk, dv = binding.uvprune_select_gather(mass[1], mass[0], 0, cfg.m, cfg.k_keep, k, v, want_score=True)
+    tl, dl, tok, u = wl.accept_inputs(cfg)
+    acc = binding.spec_accept(torch.from_numpy(tl).cuda(), torch.from_numpy(dl).cuda(),
+                              torch.from_numpy(tok).cuda(), torch.from_numpy(u).cuda())
+    torch.cuda.synchronize()
+
+    # ---- oracle
+    O_ref, L_ref, M_ref = oracle_attn(*ref_in, cfg.n_ctx)
+    O_cur, L_cur, M_cur = oracle_attn(*cur_in, cfg.n_ctx)
+    assert_o_close(o[0], O_ref)
+    assert_o_close(o[1], O_cur)
+    assert_rel_close(mass[0].cpu().numpy(), M_ref, what="mass(ref)")
+    assert_rel_close(mass[1].cpu().numpy(), M_cur, what="mass(cur)")
+    assert abs(float(mass[1].double().sum()) - cfg.Hq * cfg.R) < 1e-4 * cfg.Hq * cfg.R
+
+    # kept indices are bit-exact when computed from the GPU's own fp32 masses ...
+    g_cur, g_ref = mass[1].cpu().numpy(), mass[0].cpu().numpy()
+    np.testing.assert_array_equal(kept.cpu().numpy(), select_topk(score_fp32(g_cur, g_ref, 0, cfg.m), cfg.k_keep))
+    np.testing.assert_array_equal(score.cpu().numpy(), score_fp32(g_cur, g_ref, 0, cfg.m))
+    # ... and end to end may differ from the oracle's only where a score sits within 1e-4 relative of the k-th score
+    s_or = score_fp32(M_cur.astype(np.float32), M_ref.astype(np.float32), 0, cfg.m)
+    idx_or = select_topk(s_or, cfg.k_keep)
+    diff = np.setxor1d(kept.cpu().numpy(), idx_or)
+    tau = np.sort(s_or)[::-1][cfg.k_keep - 1]
+    for i in diff:
+        assert abs(float(s_or[i]) - float(tau)) <= 1e-4 * max(abs(float(s_or[i])), abs(float(tau)), 1e-30) + 2e-6, \
+            (i, s_or[i], tau)
+    assert diff.size <= max(4, cfg.k_keep // 100)
+
+    # gather is byte exact for the indices the GPU selected
+    idx = kept.cpu().numpy()
+    src_k = np.stack([ref_in[1], cur_in[1]])
+    src_v = np.stack([ref_in[2], cur_in[2]])
+    assert bits_of(dk).tobytes() == gather_rows(src_k, 0, cfg.m, idx).tobytes()
+    assert bits_of(dv).tobytes() == gather_rows(src_v, 0, cfg.m, idx).tobytes()
+    assert dk.shape[1] == cfg.T - cfg.m + cfg.k_keep
+
+    # accept / resample
+    r = oracle_accept(tl, dl, tok, u)
+    n_g = int(acc["n_accept"])
+    if n_g != r["n_accept"]:
+        t = min(n_g, r["n_accept"])
+        assert abs(float(u[t]) - float(r["p"][t, tok[t]] / r["q"][t, tok[t]])) <= 1e-5
+    else:
+        np.testing.assert_array_equal(acc["out_tokens"].cpu().numpy()[:n_g], tok[:n_g])
+        assert acc["out_tokens"].cpu().numpy()[n_g] == r["out_tokens"][n_g]
+
+
+def test_verify_step_host_buffers_config0():
+    """The single-call step with host inputs/outputs gives the same results as the three calls."""
+    cfg = wl.CONFIGS[0]
+    ref_in, cur_in = layers_for(cfg)
+    dev = torch.device("cuda", 0)
+    q = torch.stack([bf16_cuda(ref_in[0]), bf16_cuda(cur_in[0])])
+    k = torch.stack([bf16_cuda(ref_in[1]), bf16_cuda(cur_in[1])])
+    v = torch.stack([bf16_cuda(ref_in[2]), bf16_cuda(cur_in[2])])
+    tl, dl, tok, u = wl.accept_inputs(cfg)
+    # expected: separate calls
+    o_e, lse_e, mass_e = binding.verify_attn(q, k, v, cfg.n_ctx, want_mass=True)
+    kept_e, _, dk_e, dv_e = binding.uvprune_select_gather(mass_e[1], mass_e[0], 0, cfg.m, cfg.k_keep, k, v)
+    acc_e = binding.spec_accept(torch.from_numpy(tl).cuda(), torch.from_numpy(dl).cuda(),
+                                torch.from_numpy(tok).cuda(), torch.from_numpy(u).cuda())
+    torch.cuda.synchronize()
+    # step call: device buffers start zeroed / scrambled, inputs arrive from the host
+    q2 = torch.zeros_like(q)
+    k2, v2 = k.clone(), v.clone()
+    k2[:, cfg.n_ctx:] = 0
+    v2[:, cfg.n_ctx:] = 0
+    o2 = torch.zeros_like(q)
+    mass2 = torch.zeros((2, cfg.T), dtype=torch.float32, device=dev)
+    kept2 = torch.zeros(cfg.k_keep, dtype=torch.int32, device=dev)
+    S2 = cfg.T - cfg.m + cfg.k_keep
+    dk2 = torch.zeros((2, S2, cfg.Hkv, cfg.D), dtype=torch.bfloat16, device=dev)
+    dv2 = torch.zeros_like(dk2)
+    tl2 = torch.zeros(tl.shape, device=dev)
+    dl2 = torch.zeros(dl.shape, device=dev)
+    tok2 = torch.zeros(cfg.gamma, dtype=torch.int32, device=dev)
+    u2 = torch.zeros(cfg.gamma + 1, device=dev)
+    outs = dict(n_accept=torch.zeros(1, dtype=torch.int32, device=dev),
+                out_tokens=torch.zeros((1, cfg.gamma + 1), dtype=torch.int32, device=dev))
+    pa = binding.attn_params(q2, k2, v2, cfg.n_ctx, o2, None, mass2)
+    pp = binding.prune_params(mass2[1], mass2[0], 0, cfg.m, cfg.k_keep, kept2, None, k2, v2, dk2, dv2)
+    pc = binding.accept_params(tl2, dl2, tok2, u2, 1.0, outs)
+    pin = lambda t: t.contiguous().cpu().pin_memory()
+    h_in = dict(h_q=pin(q), h_k_window=pin(k[:, cfg.n_ctx:]), h_v_window=pin(v[:, cfg.n_ctx:]),
+                h_target_logits=torch.from_numpy(tl).pin_memory(), h_draft_logits=torch.from_numpy(dl).pin_memory(),
+                h_draft_tokens=torch.from_numpy(tok).pin_memory(), h_uniforms=torch.from_numpy(u).pin_memory())
+    h_out = dict(h_o=torch.zeros(q.shape, dtype=torch.bfloat16).pin_memory(),
+                 h_n_accept=torch.zeros(1, dtype=torch.int32).pin_memory(),
+                 h_out_tokens=torch.zeros(cfg.gamma + 1, dtype=torch.int32).pin_memory(),
+                 h_kept_idx=torch.zeros(cfg.k_keep, dtype=torch.int32).pin_memory())
+    binding.verify_step(pa, pp, pc, host_in=h_in, host_out=h_out)
+    torch.cuda.synchronize()
+    assert torch.equal(h_out["h_o"], o_e.cpu())
+    assert torch.equal(k2, k) and torch.equal(v2, v)                     # window rows landed in the cache
+    assert torch.equal(h_out["h_kept_idx"], kept_e.cpu())
+    assert torch.equal(dk2, dk_e) and torch.equal(dv2, dv_e)
+    assert int(h_out["h_n_accept"]) == int(acc_e["n_accept"])
+    assert torch.equal(h_out["h_out_tokens"], acc_e["out_tokens"].cpu())
+
+
+def test_draft_and_verify_streams_run_concurrently_and_agree():
+    """Draft-side decode attention (R = 1 over the compacted cache) on one stream while the
+    verify pass runs on another: each stream has its own workspace; results equal the
+    serial ones bit for bit."""
+    cfg = wl.CONFIGS[0]
+    q, k, v = (bf16_cuda(x) for x in wl.attn_layer(cfg, 0))
+    qd, kd, vd = (bf16_cuda(x) for x in wl.make_qkv(8, 2, 64, 1, 400, sink=False, seed=77))
+    o_s, lse_s, mass_s = binding.verify_attn(q, k, v, cfg.n_ctx, want_mass=True)
+    od_s, lsed_s, _ = binding.verify_attn(qd, kd, vd, 399)
+    torch.cuda.synchronize()
+    sv, sd = torch.cuda.Stream(), torch.cuda.Stream()
+    for _ in range(5):
+        with torch.cuda.stream(sv):
+            o_c, lse_c, mass_c = binding.verify_attn(q, k, v, cfg.n_ctx, want_mass=True)
+        with torch.cuda.stream(sd):
+            od_c, lsed_c, _ = binding.verify_attn(qd, kd, vd, 399)
+    torch.cuda.synchronize()
+    assert torch.equal(o_c, o_s) and torch.equal(mass_c, mass_s) and torch.equal(lse_c, lse_s)
+    assert torch.equal(od_c, od_s) and torch.equal(lsed_c, lsed_s)
