@@ -37,7 +37,8 @@ enum {
   PVLM_ERR_INVALID_ARG = 1, /* NULL where data is required, negative size, bad stride or alignment */
   PVLM_ERR_UNSUPPORTED = 2, /* shape outside the compiled set (see each call) */
   PVLM_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned or too small */
-  PVLM_ERR_CUDA = 4         /* a launch failed; see pvlm_last_cuda_error() */
+  PVLM_ERR_CUDA = 4,        /* a launch failed; see pvlm_last_cuda_error() */
+  PVLM_ERR_TOO_LARGE = 5    /* size beyond the fixed capacity of a no-allocation entry point */
 };
 
 /* Human-readable name of a status code (static storage). */
@@ -217,6 +218,45 @@ typedef struct {
 } pvlm_step_params;
 
 pvlm_status pvlm_verify_step(const pvlm_step_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Top-K selection that needs no caller-side scratch allocation.
+ * (The paper has no counterpart: this is a packaging variant of the
+ * selection half of pvlm_uvprune_select_gather, for callers that cannot
+ * allocate device memory.)
+ *
+ * Some callers of this library cannot call cudaMalloc at the point where
+ * they need a selection: code running inside a pre-sized memory arena whose
+ * budget is fixed at start-up, plug-ins loaded into a host process that owns
+ * all device memory, or a latency-critical loop where an allocation (which
+ * may synchronise the device) is not acceptable.  pvlm_uvprune_select_gather
+ * asks such a caller for a workspace it has no way to provide.  This entry
+ * point computes exactly the same kept_idx (same score, same tie rule, same
+ * ascending order) but keeps its scratch (one 32-bit key per visual token) in
+ * a fixed array inside the library's device image.
+ *
+ * Capacity: m <= PVLM_SELECT_STATIC_MAX_M.  A larger m returns
+ * PVLM_ERR_TOO_LARGE and launches nothing.  The array costs
+ * 4 * PVLM_SELECT_STATIC_MAX_M bytes (1 MiB) of device memory on every GPU
+ * that loads the library, from load until process exit.
+ *
+ * The call allocates nothing and frees nothing, on host or device.  The first
+ * call on each device looks up the array's device address (a driver query, no
+ * allocation); make that first call outside any CUDA stream capture.
+ *
+ * All calls on one device share the one array.  Nothing in it has to start at
+ * zero: every call overwrites the first m keys before reading them, so what
+ * an earlier call left behind is never observed.  Two calls that may run on
+ * the GPU at the same time (different streams without an ordering between
+ * them) race on the array and give undefined kept_idx; order them on one
+ * stream or with events.
+ *
+ * mass_cur, mass_ref, vis_start, m, k, kept_idx, score: as in pvlm_prune_params
+ * (mass_ref and score nullable).  No gather is performed.
+ * ---------------------------------------------------------------------- */
+#define PVLM_SELECT_STATIC_MAX_M 262144
+pvlm_status pvlm_uvprune_select_static(const float *mass_cur, const float *mass_ref, int vis_start, int m, int k,
+                                       int *kept_idx, float *score, void *stream);
 
 #ifdef __cplusplus
 }

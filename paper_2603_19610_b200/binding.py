@@ -19,7 +19,8 @@ _LIB = None
 _LOCK = threading.Lock()
 
 STATUS_NAMES = {0: "PVLM_OK", 1: "PVLM_ERR_INVALID_ARG", 2: "PVLM_ERR_UNSUPPORTED",
-                3: "PVLM_ERR_WORKSPACE", 4: "PVLM_ERR_CUDA"}
+                3: "PVLM_ERR_WORKSPACE", 4: "PVLM_ERR_CUDA", 5: "PVLM_ERR_TOO_LARGE"}
+SELECT_STATIC_MAX_M = 262144
 
 
 class PvlmError(RuntimeError):
@@ -77,7 +78,8 @@ class StepParams(C.Structure):
 EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
            "pvlm_verify_attn_workspace_bytes", "pvlm_verify_attn",
            "pvlm_uvprune_workspace_bytes", "pvlm_uvprune_select_gather",
-           "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept", "pvlm_verify_step")
+           "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept", "pvlm_verify_step",
+           "pvlm_uvprune_select_static")
 
 
 def lib() -> C.CDLL:
@@ -100,6 +102,9 @@ def lib() -> C.CDLL:
                 f = getattr(L, name)
                 f.restype = C.c_int
                 f.argtypes = [C.POINTER(st), C.c_void_p]
+            L.pvlm_uvprune_select_static.restype = C.c_int
+            L.pvlm_uvprune_select_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                                     C.c_void_p, C.c_void_p, C.c_void_p]
             _LIB = L
     return _LIB
 
@@ -313,3 +318,17 @@ def verify_step(attn: AttnParams | None, prune: PruneParams | None, accept: Acce
         raise PvlmError(st, "pvlm_verify_step")
     sp._keep = keep
     return sp
+
+
+def uvprune_select_static(mass_cur, mass_ref, vis_start: int, m: int, k: int, kept_idx, score=None):
+    """Top-K selection through pvlm_uvprune_select_static, the entry point for callers that
+    cannot allocate device memory: the library's built-in key buffer is the only scratch and
+    the call itself allocates nothing, so the caller passes the output tensors
+    (kept_idx int32 [k], optionally score fp32 [m]).  m is limited to SELECT_STATIC_MAX_M;
+    calls that may overlap on the GPU share the buffer and must be ordered."""
+    _need_cuda(mass_cur, mass_ref, kept_idx, score)
+    st = lib().pvlm_uvprune_select_static(_ptr(mass_cur), _ptr(mass_ref), vis_start, m, k, _ptr(kept_idx),
+                                          _ptr(score), _stream(mass_cur.device))
+    if st != 0:
+        raise PvlmError(st, "pvlm_uvprune_select_static")
+    return kept_idx

@@ -37,6 +37,7 @@ const char* pvlm_status_string(pvlm_status s) {
     case PVLM_ERR_UNSUPPORTED: return "PVLM_ERR_UNSUPPORTED";
     case PVLM_ERR_WORKSPACE: return "PVLM_ERR_WORKSPACE";
     case PVLM_ERR_CUDA: return "PVLM_ERR_CUDA";
+    case PVLM_ERR_TOO_LARGE: return "PVLM_ERR_TOO_LARGE";
     default: return "PVLM_ERR_UNKNOWN";
   }
 }

@@ -2,6 +2,7 @@
 // lower-index tie break, ascending output) and the row gather that builds the
 // compacted draft cache.
 #include "pvlm_common.cuh"
+#include <mutex>
 
 namespace pvlm {
 
@@ -178,4 +179,56 @@ pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s) {
   return check_launch();
 }
 
+// ---- selection without caller-provided scratch -------------------------------------------
+// The key buffer of the selection kernel, held in the library's device image so that callers
+// who cannot allocate device memory can still select.  In host code this name is only a
+// handle for the symbol: the kernel must be given the address cudaGetSymbolAddress returns.
+static __device__ __align__(256) uint32_t g_select_static_keys[PVLM_SELECT_STATIC_MAX_M];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+uint32_t* g_static_keys_addr[kMaxDevices] = {};
+
+// Device address of the static key buffer on the current device; looked up once per device.
+pvlm_status static_keys_for_current_device(uint32_t** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+  if (dev < 0 || dev >= kMaxDevices) return PVLM_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_keys_addr[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_select_static_keys);
+    if (e != cudaSuccess || !ptr) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+    g_static_keys_addr[dev] = static_cast<uint32_t*>(ptr);
+  }
+  *out = g_static_keys_addr[dev];
+  return PVLM_OK;
+}
+}  // namespace
+
 }  // namespace pvlm
+
+extern "C" pvlm_status pvlm_uvprune_select_static(const float* mass_cur, const float* mass_ref, int vis_start, int m,
+                                                  int k, int* kept_idx, float* score, void* stream) {
+  using namespace pvlm;
+  if (m < 0 || k < 0 || k > m || vis_start < 0) return PVLM_ERR_INVALID_ARG;
+  if (m > PVLM_SELECT_STATIC_MAX_M) return PVLM_ERR_TOO_LARGE;
+  if (m > 0 && !mass_cur) return PVLM_ERR_INVALID_ARG;
+  if (k > 0 && !kept_idx) return PVLM_ERR_INVALID_ARG;
+  if (m == 0) return PVLM_OK;
+  uint32_t* keys = nullptr;
+  const pvlm_status st = static_keys_for_current_device(&keys);
+  if (st != PVLM_OK) return st;
+  SelArgs sa;
+  sa.cur = mass_cur + vis_start;
+  sa.ref = mass_ref ? mass_ref + vis_start : nullptr;
+  sa.score = score;
+  sa.keys = keys;
+  sa.kept = kept_idx;
+  sa.m = m;
+  sa.k = k;
+  uvprune_select_kernel<<<1, kSelThreads, 0, (cudaStream_t)stream>>>(sa);
+  return check_launch();
+}
