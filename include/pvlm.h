@@ -38,7 +38,8 @@ enum {
   PVLM_ERR_UNSUPPORTED = 2, /* shape outside the compiled set (see each call) */
   PVLM_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned or too small */
   PVLM_ERR_CUDA = 4,        /* a launch failed; see pvlm_last_cuda_error() */
-  PVLM_ERR_TOO_LARGE = 5    /* size beyond the fixed capacity of a no-allocation entry point */
+  PVLM_ERR_TOO_LARGE = 5,   /* size beyond the fixed capacity of a no-allocation entry point */
+  PVLM_ERR_TIMEOUT = 6      /* a bounded on-device wait expired; outputs of that call are undefined */
 };
 
 /* Human-readable name of a status code (static storage). */
@@ -98,6 +99,11 @@ typedef struct {
 /* Host-only; needs no GPU.  Returns 0 if the parameters are unsupported. */
 size_t pvlm_verify_attn_workspace_bytes(const pvlm_attn_params *p);
 pvlm_status pvlm_verify_attn(const pvlm_attn_params *p, void *stream);
+/* Health check of the last pvlm_verify_attn issued with this parameter block (same workspace):
+ * every wait inside the kernels is bounded, and one that expires records it in the workspace
+ * instead of hanging.  This call SYNCHRONISES `stream`, reads that word and returns PVLM_OK or
+ * PVLM_ERR_TIMEOUT.  Optional: results of a call that timed out are undefined either way. */
+pvlm_status pvlm_verify_attn_check(const pvlm_attn_params *p, void *stream);
 
 /* ------------------------------------------------------------------------
  * UV-Prune: debiased score, Top-K selection, gather into the draft cache.

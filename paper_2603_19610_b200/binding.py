@@ -19,7 +19,7 @@ _LIB = None
 _LOCK = threading.Lock()
 
 STATUS_NAMES = {0: "PVLM_OK", 1: "PVLM_ERR_INVALID_ARG", 2: "PVLM_ERR_UNSUPPORTED",
-                3: "PVLM_ERR_WORKSPACE", 4: "PVLM_ERR_CUDA", 5: "PVLM_ERR_TOO_LARGE"}
+                3: "PVLM_ERR_WORKSPACE", 4: "PVLM_ERR_CUDA", 5: "PVLM_ERR_TOO_LARGE", 6: "PVLM_ERR_TIMEOUT"}
 SELECT_STATIC_MAX_M = 262144
 
 
@@ -76,7 +76,7 @@ class StepParams(C.Structure):
 
 
 EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
-           "pvlm_verify_attn_workspace_bytes", "pvlm_verify_attn",
+           "pvlm_verify_attn_workspace_bytes", "pvlm_verify_attn", "pvlm_verify_attn_check",
            "pvlm_uvprune_workspace_bytes", "pvlm_uvprune_select_gather",
            "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept", "pvlm_verify_step",
            "pvlm_uvprune_select_static")
@@ -98,7 +98,8 @@ def lib() -> C.CDLL:
                 f.restype = C.c_size_t
                 f.argtypes = [C.POINTER(st)]
             for name, st in (("pvlm_verify_attn", AttnParams), ("pvlm_uvprune_select_gather", PruneParams),
-                             ("pvlm_spec_accept", AcceptParams), ("pvlm_verify_step", StepParams)):
+                             ("pvlm_spec_accept", AcceptParams), ("pvlm_verify_step", StepParams),
+                             ("pvlm_verify_attn_check", AttnParams)):
                 f = getattr(L, name)
                 f.restype = C.c_int
                 f.argtypes = [C.POINTER(st), C.c_void_p]
@@ -166,7 +167,7 @@ def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None, mass_la
 
 
 def verify_attn(q, k, v, n_ctx: int, *, want_lse: bool = True, want_mass: bool = False, scale: float = 0.0,
-                out=None, workspace=None, mass_layers=None):
+                out=None, workspace=None, mass_layers=None, check: bool = False):
     """Window-verify GQA attention (see pvlm_verify_attn).  Returns (o, lse, mass).
 
     mass_layers (batched form only): list of layer indices whose mass is wanted;
@@ -184,6 +185,10 @@ def verify_attn(q, k, v, n_ctx: int, *, want_lse: bool = True, want_mass: bool =
     st = lib().pvlm_verify_attn(C.byref(p), _stream(q.device))
     if st != 0:
         raise PvlmError(st, "pvlm_verify_attn")
+    if check:                                    # synchronises: did any bounded on-device wait expire?
+        st = lib().pvlm_verify_attn_check(C.byref(p), _stream(q.device))
+        if st != 0:
+            raise PvlmError(st, "pvlm_verify_attn_check")
     return o, lse, mass
 
 

@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libpvlm.so")
-SOURCES = ["pvlm_api.cu", "verify_attn.cu", "uvprune.cu", "spec_accept.cu"]
+SOURCES = ["pvlm_api.cu", "verify_attn.cu", "verify_attn_tc.cu", "uvprune.cu", "spec_accept.cu"]
 
 
 def _nvcc() -> str:
@@ -33,7 +33,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB_PATH
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-lcuda",
            "-o", LIB_PATH] + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")

@@ -38,6 +38,7 @@ const char* pvlm_status_string(pvlm_status s) {
     case PVLM_ERR_WORKSPACE: return "PVLM_ERR_WORKSPACE";
     case PVLM_ERR_CUDA: return "PVLM_ERR_CUDA";
     case PVLM_ERR_TOO_LARGE: return "PVLM_ERR_TOO_LARGE";
+    case PVLM_ERR_TIMEOUT: return "PVLM_ERR_TIMEOUT";
     default: return "PVLM_ERR_UNKNOWN";
   }
 }
@@ -79,6 +80,22 @@ pvlm_status pvlm_verify_attn(const pvlm_attn_params* p, void* stream) {
   const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, plan.total);
   if (w != PVLM_OK) return w;
   return launch_verify_attn(*p, plan, (cudaStream_t)stream);
+}
+
+pvlm_status pvlm_verify_attn_check(const pvlm_attn_params* p, void* stream) {
+  if (!p) return PVLM_ERR_INVALID_ARG;
+  AttnPlan plan;
+  if (!make_attn_plan(*p, plan)) return PVLM_ERR_UNSUPPORTED;
+  const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, plan.total);
+  if (w != PVLM_OK) return w;
+  int word = 0;
+  cudaError_t e = cudaSuccess;
+  if (plan.use_tc)
+    e = cudaMemcpyAsync(&word, (const char*)p->workspace + plan.off_tc + plan.tc.off_status, 4, cudaMemcpyDeviceToHost,
+                        (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+  return word ? PVLM_ERR_TIMEOUT : PVLM_OK;
 }
 
 size_t pvlm_uvprune_workspace_bytes(const pvlm_prune_params* p) {

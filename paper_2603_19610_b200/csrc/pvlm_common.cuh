@@ -22,7 +22,19 @@ void set_cuda_error(int e);
 // ---- verify attention -----------------------------------------------------
 constexpr int kAttnBN = 64;           // keys per tile
 
+struct AttnTcPlan {           // tensor-core (tcgen05) path, D = 128
+  int nrp;                    // query rows per KV head padded to a multiple of 16
+  int T, tiles_per_item, n_cta, seg_max;
+  long long total_tiles;
+  size_t off_part_o, off_part_ml, off_status, total;   // relative to the path's workspace region
+};
+bool make_attn_tc_plan(const pvlm_attn_params& p, AttnTcPlan& plan);
+pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& plan, char* ws, float* lse2, cudaStream_t s);
+
 struct AttnPlan {
+  bool use_tc;     // main pass on tcgen05; the mma.sync kernel still runs the mass pass
+  AttnTcPlan tc;
+  size_t off_tc;
   int rows;        // G * R valid rows per KV head
   int n_warps;     // 16-row MMA tiles (one warp each)
   int rows_pad;    // n_warps * 16

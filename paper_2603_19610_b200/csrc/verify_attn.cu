@@ -9,6 +9,9 @@
 // different normalisers and cannot be rescaled after the fact.
 #include "pvlm_common.cuh"
 
+#include <cstdlib>
+#include <cstring>
+
 namespace pvlm {
 
 namespace {
@@ -357,8 +360,10 @@ pvlm_status launch_dw(const AttnArgs& a, const pvlm_attn_params& p, const AttnPl
   const int smem0 = kStages * 2 * kAttnBN * D * 2;
   cudaFuncSetAttribute(attn_kernel<D, 0, MAXW>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0);
   cudaFuncSetAttribute(attn_kernel<D, 0, MAXW>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-  attn_kernel<D, 0, MAXW><<<grid, threads, smem0, s>>>(a);
-  if (plan.splits > 1) attn_combine_kernel<D><<<dim3(plan.rows, p.Hkv, p.n_layers), D, 0, s>>>(a);
+  if (!plan.use_tc) {
+    attn_kernel<D, 0, MAXW><<<grid, threads, smem0, s>>>(a);
+    if (plan.splits > 1) attn_combine_kernel<D><<<dim3(plan.rows, p.Hkv, p.n_layers), D, 0, s>>>(a);
+  }
   if (p.mass) {
     const int smem1 = kStages * kAttnBN * D * 2 + 8 * kAttnBN * 4;
     cudaFuncSetAttribute(attn_kernel<D, 1, MAXW>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1);
@@ -404,6 +409,11 @@ bool make_attn_plan(const pvlm_attn_params& p, AttnPlan& plan) {
     const int n_mass = p.mass_layers ? p.n_mass_layers : p.n_layers;
     off += align_up((size_t)n_mass * p.Hkv * align_up(plan.T, kAttnBN) * 4, 256);
   }
+  // main pass on the tcgen05 kernel whenever it applies (PVLM_ATTN_IMPL=mma forces the mma.sync kernel)
+  const char* impl = getenv("PVLM_ATTN_IMPL");
+  plan.use_tc = (p.D == 128) && !(impl && strcmp(impl, "mma") == 0) && make_attn_tc_plan(p, plan.tc);
+  plan.off_tc = off;
+  if (plan.use_tc) off += align_up(plan.tc.total, 256);
   plan.total = off;
   return true;
 }
@@ -432,6 +442,11 @@ pvlm_status launch_verify_attn(const pvlm_attn_params& p, const AttnPlan& plan, 
   a.mass_listed = p.mass_layers != nullptr;
   a.n_mass = a.mass_listed ? p.n_mass_layers : p.n_layers;
   for (int i = 0; i < 8; ++i) a.mass_layer[i] = (a.mass_listed && i < p.n_mass_layers) ? p.mass_layers[i] : 0;
+  if (plan.use_tc) {
+    const pvlm_status st = launch_verify_attn_tc(p, plan.tc, ws + plan.off_tc, a.lse2, s);
+    if (st != PVLM_OK) return st;
+    if (!p.mass) return PVLM_OK;
+  }
   return p.D == 64 ? launch_d<64>(a, p, plan, s) : launch_d<128>(a, p, plan, s);
 }
 
