@@ -87,7 +87,7 @@ def lib() -> C.CDLL:
     global _LIB
     with _LOCK:
         if _LIB is None:
-            path = _build.build()
+            path = os.environ.get("PVLM_LIB") or _build.build()     # PVLM_LIB: use a library built elsewhere
             L = C.CDLL(path)
             L.pvlm_status_string.restype = C.c_char_p
             L.pvlm_status_string.argtypes = [C.c_int]

@@ -5,15 +5,18 @@
 // contiguous range segment by segment (a segment = its tiles of one item).  Every segment ends in a
 // partial (O, m, l) written to the workspace; a small combine kernel merges an item's segments.
 //
-// Inside a CTA (10 warps):
-//   warp 0      TMA producer: K and V tiles (two 64-channel boxes each, 128-byte swizzle) into
-//               separate 2-deep shared-memory rings, completion on mbarriers.
-//   warp 1      MMA issuer (one thread): S^T = K . Q^T  (M = 128 keys, N = padded query rows,
-//               K = 128 channels) into one of two TMEM score buffers, then O^T += V^T . P^T
-//               (M = 128 channels, N = rows, K = 128 keys) into the TMEM output accumulator.
-//   warps 2..9  softmax: each thread owns one key (TMEM lane) and half of the query-row columns,
-//               so exp2, the running row sums and the bf16 pack are thread-local; P is written to
-//               shared memory in the MN-major core-matrix layout the second MMA reads.
+// Inside a CTA (12 warps = 3 warpgroups; registers are moved from warpgroup 0 to the softmax
+// warpgroups with setmaxnreg):
+//   warp 0       TMA producer: K and V tiles (two 64-channel boxes each, 128-byte swizzle) into
+//                separate 2-deep shared-memory rings, completion on mbarriers.
+//   warp 1       MMA issuer (one thread): S^T = K . Q^T  (M = 128 keys, N = padded query rows,
+//                K = 128 channels) into one of up to four TMEM score buffers, then O^T += V^T . P^T
+//                (M = 128 channels, N = rows, K = 128 keys) into a TMEM output accumulator.
+//   warps 4..11  two softmax groups working on alternate tiles, each with its own accumulator,
+//                reference and row sums (two interleaved online-softmax streams).  A thread owns
+//                one key (TMEM lane) of its group's tile and all query-row columns, so exp2, the
+//                running row sums and the bf16 pack are thread-local; P is written to shared
+//                memory in the MN-major core-matrix layout the second MMA reads.
 // The transposed orientation keeps all 128 TMEM lanes busy although only G*R <= 128 (typically
 // 65..88) query rows exist, and makes N (not M) the padded dimension: N = 80 instead of M = 128.
 //
@@ -25,18 +28,19 @@
 
 #include <cuda.h>
 
+#include <cstdlib>
+
 namespace pvlm {
 
 namespace {
 
 constexpr int kTile = 128;                 // keys per tile
 constexpr int kKStages = 2, kVStages = 2;
-// P buffers: two, except for the widest row counts where shared memory only has room for one
-__host__ __device__ constexpr int p_bufs(int nrp) { return nrp > 96 ? 1 : 2; }
 constexpr int kBoxBytes = kTile * 128;     // one 64-channel box of a 128-key tile: 16 KB
 constexpr int kTileBytes = 2 * kBoxBytes;  // 32 KB
 constexpr int kSoftmaxThreads = 256;
-constexpr int kThreads = 64 + kSoftmaxThreads;
+constexpr int kGroupThreads = 128;         // one softmax group
+constexpr int kThreads = 128 + kSoftmaxThreads;   // warpgroup 0: TMA + MMA (+2 idle warps); warpgroups 1, 2: softmax
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 constexpr float kNegBig = -1.0e30f;        // "no key seen yet" reference: finite, so differences never give NaN
@@ -52,6 +56,7 @@ struct TcArgs {
   long long total_tiles;     // W = items * Tt
   int seg_max;               // partial slots per CTA
   int n_cta;
+  uint32_t g_magic;          // ceil(2^16 / G): row / G == (row * g_magic) >> 16 for row < 128
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -99,22 +104,27 @@ __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr));
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
 }
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
-               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-               : "memory");
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+// Makes the compiler treat the registers as written here, i.e. after the preceding wait::ld.
+__device__ __forceinline__ void reg_fence16(uint32_t (&r)[16]) {
+  asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                    "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]));
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// Makes the compiler treat the registers as written here, i.e. after the preceding wait::ld.
-__device__ __forceinline__ void reg_fence8(uint32_t (&r)[8]) {
-  asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]));
-}
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
@@ -130,13 +140,12 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
 }
-__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ bool softmax_bar_or(bool pred) {
   uint32_t out;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\t"
       "setp.ne.u32 p, %1, 0;\n\t"
-      "bar.red.or.pred q, 1, 256, p;\n\t"
+      "bar.red.or.pred q, 3, 256, p;\n\t"
       "selp.u32 %0, 1, 0, q;\n\t}"
       : "=r"(out)
       : "r"((uint32_t)pred)
@@ -156,35 +165,52 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
          (1ull << 46) | ((uint64_t)layout << 61);
 }
 
+#ifdef PVLM_TC_PROFILE
+#define PROF_DECL long long prof_t0 = 0; long long prof_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+#define PROF_START prof_t0 = clock64();
+#define PROF_ADD(i) { const long long now = clock64(); prof_acc[i] += now - prof_t0; prof_t0 = now; }
+#define PROF_DUMP(base) { for (int pi = 0; pi < 12; ++pi) a.status[(base) + pi] = (int)(prof_acc[pi] >> 4); }
+#else
+#define PROF_DECL
+#define PROF_START
+#define PROF_ADD(i)
+#define PROF_DUMP(base) {}
+#endif
+
 // ---------------------------------------------------------------------------------------------
-// The kernel.  NRP = query rows per KV head padded to a multiple of 16 (MMA N).
+// The kernel.  NRP = query rows per KV head padded to a multiple of 16 (MMA N), NRP <= 96.
 // ---------------------------------------------------------------------------------------------
+__host__ __device__ constexpr int s_bufs(int nrp) { return (512 - 2 * nrp) / nrp >= 4 ? 4 : (512 - 2 * nrp) / nrp; }
+
 template <int NRP>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const TcArgs a) {
-  constexpr int HALF = NRP / 2;            // columns per softmax thread
-  constexpr int NCH = HALF / 8;            // 8-column chunks per thread
+  constexpr int NCH = NRP / 16;            // 16-column chunks per thread
   constexpr int QBOX = NRP * 128;          // bytes of one 64-channel box of Q
   constexpr int PBYTES = NRP * 256;        // one P buffer: NRP/8 row groups x 2048 B
-  constexpr int kPBufs = p_bufs(NRP);
-  constexpr uint32_t TMEM_COLS = (3 * NRP <= 32) ? 32 : (3 * NRP <= 64) ? 64 : (3 * NRP <= 128) ? 128 : (3 * NRP <= 256) ? 256 : 512;
+  constexpr int NSB = s_bufs(NRP);         // score buffers in TMEM
+  constexpr uint32_t NEED = (2 + NSB) * NRP;
+  constexpr uint32_t TMEM_COLS = NEED <= 32 ? 32 : NEED <= 64 ? 64 : NEED <= 128 ? 128 : NEED <= 256 ? 256 : 512;
   constexpr uint32_t IDESC_QK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NRP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   constexpr uint32_t IDESC_PV = IDESC_QK | (1u << 15) | (1u << 16);
+  static_assert(NRP % 16 == 0 && NRP <= 96 && NSB >= 2, "row padding");
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned char* sK = smem;
   unsigned char* sV = sK + kKStages * kTileBytes;
   unsigned char* sQ = sV + kVStages * kTileBytes;
-  unsigned char* sP = sQ + 2 * QBOX;
-  int* s_newmax = reinterpret_cast<int*>(sP + kPBufs * PBYTES);      // [128]
-  float* s_lsum = reinterpret_cast<float*>(s_newmax + 128);          // [4][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(s_lsum + 4 * 128);
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 24);
+  unsigned char* sP = sQ + 2 * QBOX;                                  // one P buffer per softmax group
+  float* s_m = reinterpret_cast<float*>(sP + 2 * PBYTES);            // [2][128] running reference per group
+  float* s_fac = s_m + 256;                                           // [2][128] rescale factors (slow path)
+  int* s_newmax = reinterpret_cast<int*>(s_fac + 256);               // [2][128]
+  float* s_lsum = reinterpret_cast<float*>(s_newmax + 256);          // [2][4][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_lsum + 1024);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
-  enum { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_FREE = 10, P_FULL = 12, P_FREE = 14,
-         Q_READY = 16, O_FULL = 17, O_FREE = 18 };
+  enum { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, P_FULL = 8, P_FREE = 10, Q_READY = 12, O_FULL = 13, O_FREE = 14,
+         S_FULL = 16, S_FREE = 20 };
   auto bar = [&](int i) { return smem_addr(bars + i); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -199,9 +225,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1);
       mbar_init(bar(V_FULL + i), 1); mbar_init(bar(V_EMPTY + i), 1);
-      mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), kSoftmaxThreads);
-      mbar_init(bar(P_FULL + i), kSoftmaxThreads); mbar_init(bar(P_FREE + i), 1);
+      mbar_init(bar(P_FULL + i), kGroupThreads); mbar_init(bar(P_FREE + i), 1);
     }
+    for (int i = 0; i < NSB; ++i) { mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), kGroupThreads); }
     mbar_init(bar(Q_READY), kSoftmaxThreads);
     mbar_init(bar(O_FULL), 1);
     mbar_init(bar(O_FREE), kSoftmaxThreads);
@@ -214,53 +240,95 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   }
   // zero Q (its padding rows are never written again) and the slow-path scratch
   for (int i = tid; i < 2 * QBOX / 16; i += kThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
-  if (tid < 128) s_newmax[tid] = f2ord(-INFINITY);
+  if (tid < 256) s_newmax[tid] = f2ord(-INFINITY);
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
-  const uint32_t tmem_S0 = tmem, tmem_O = tmem + 2 * NRP;
+  const uint32_t tmem_O = tmem;                    // O accumulators of the two softmax groups: columns [g*NRP, (g+1)*NRP)
+  const uint32_t tmem_S = tmem + 2 * NRP;          // score buffers
 
   if (f_end > f_begin) {
+    if (warp < 4) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == 0) {
       // =========================== TMA producer ===========================
       if (lane == 0) {
-        uint32_t jt = 0;
-        for (long long f = f_begin; f < f_end; ++f, ++jt) {
-          const int item = (int)(f / Tt), tile = (int)(f - (long long)item * Tt);
-          const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
-          const uint32_t ks = jt % kKStages, vs = jt % kVStages;
-          if (jt >= kKStages && !mbar_wait(bar(K_EMPTY + ks), ((jt / kKStages) - 1) & 1, s_abort)) break;
-          mbar_expect_tx(bar(K_FULL + ks), kTileBytes);
-          tma_load_4d(smem_addr(sK + ks * kTileBytes), &tm_k, bar(K_FULL + ks), 0, kvh, tile * kTile, layer);
-          tma_load_4d(smem_addr(sK + ks * kTileBytes + kBoxBytes), &tm_k, bar(K_FULL + ks), 64, kvh, tile * kTile, layer);
-          if (jt >= kVStages && !mbar_wait(bar(V_EMPTY + vs), ((jt / kVStages) - 1) & 1, s_abort)) break;
+        PROF_DECL
+        // K runs ahead of V by the MMA issuer's look-ahead, so the two rings advance separately:
+        // all K tiles first up to the ring depth, then alternate.
+        uint32_t jk = 0, jv = 0;
+        const uint32_t total = (uint32_t)(f_end - f_begin);
+        auto coords = [&](uint32_t j, int& kvh, int& tile, int& layer) {
+          const long long f = f_begin + j;
+          const int item = (int)(f / Tt);
+          tile = (int)(f - (long long)item * Tt);
+          layer = item / a.Hkv;
+          kvh = item - layer * a.Hkv;
+        };
+        // The MMA issuer runs the score MMAs NSB-1 tiles ahead of the PV MMAs, so V(j) may only be
+        // waited for once K has been issued through tile j+NSB-1 (otherwise the issuer would wait for
+        // a K tile that this thread, blocked on a V slot, never sends).
+        while (jk < total || jv < total) {
+          PROF_START
+          // K tiles that must be on their way before PV(jv) can be issued; never past the end of
+          // jv's segment, because the next segment's score MMAs wait for this segment's epilogue
+          uint32_t need_k = total;
+          if (jv < total) {
+            const long long fv = f_begin + jv;
+            const long long seg_end_j = min(f_end, (fv / Tt + 1) * (long long)Tt) - f_begin;
+            need_k = (uint32_t)min((long long)jv + NSB, seg_end_j);
+          }
+          if (jk < total && jk < need_k) {
+            const uint32_t ks = jk % kKStages;
+            int kvh, tile, layer;
+            coords(jk, kvh, tile, layer);
+            if (jk >= kKStages && !mbar_wait(bar(K_EMPTY + ks), ((jk / kKStages) - 1) & 1, s_abort)) break;
+            PROF_ADD(0)
+            mbar_expect_tx(bar(K_FULL + ks), kTileBytes);
+            tma_load_4d(smem_addr(sK + ks * kTileBytes), &tm_k, bar(K_FULL + ks), 0, kvh, tile * kTile, layer);
+            tma_load_4d(smem_addr(sK + ks * kTileBytes + kBoxBytes), &tm_k, bar(K_FULL + ks), 64, kvh, tile * kTile, layer);
+            ++jk;
+            continue;
+          }
+          const uint32_t vs = jv % kVStages;
+          int kvh, tile, layer;
+          coords(jv, kvh, tile, layer);
+          if (jv >= kVStages && !mbar_wait(bar(V_EMPTY + vs), ((jv / kVStages) - 1) & 1, s_abort)) break;
+          PROF_ADD(1)
           mbar_expect_tx(bar(V_FULL + vs), kTileBytes);
           tma_load_4d(smem_addr(sV + vs * kTileBytes), &tm_v, bar(V_FULL + vs), 0, kvh, tile * kTile, layer);
           tma_load_4d(smem_addr(sV + vs * kTileBytes + kBoxBytes), &tm_v, bar(V_FULL + vs), 64, kvh, tile * kTile, layer);
+          ++jv;
+          PROF_ADD(2)
         }
+        if (blockIdx.x == 0) PROF_DUMP(4)
       }
     } else if (warp == 1) {
       // =========================== MMA issuer ===========================
       if (lane == 0) {
         const uint32_t q_base = smem_addr(sQ);
         bool ok = true;
+        PROF_DECL
         uint32_t jt = 0;           // tiles issued by this CTA so far (ring phases run across segments)
         int seg = 0;
         auto issue_qk = [&](uint32_t j) -> bool {
-          const uint32_t ks = j % kKStages, sb = j & 1;
+          const uint32_t ks = j % kKStages, sb = j % NSB;
+          PROF_START
           if (!mbar_wait(bar(K_FULL + ks), (j / kKStages) & 1, s_abort)) return false;
-          if (j >= 2 && !mbar_wait(bar(S_FREE + sb), ((j >> 1) - 1) & 1, s_abort)) return false;
+          PROF_ADD(0)
+          if (j >= NSB && !mbar_wait(bar(S_FREE + sb), ((j / NSB) - 1) & 1, s_abort)) return false;
+          PROF_ADD(1)
           tc_fence_after();
           const uint32_t k_base = smem_addr(sK + ks * kTileBytes);
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) {
             const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32, qoff = (kk >> 2) * QBOX + (kk & 3) * 32;
-            tc_mma(tmem_S0 + sb * NRP, make_desc(k_base + off, 16, 1024, 2), make_desc(q_base + qoff, 16, 1024, 2), IDESC_QK, kk > 0);
+            tc_mma(tmem_S + sb * NRP, make_desc(k_base + off, 16, 1024, 2), make_desc(q_base + qoff, 16, 1024, 2), IDESC_QK, kk > 0);
           }
           tc_commit(bar(S_FULL + sb));
           tc_commit(bar(K_EMPTY + ks));
+          PROF_ADD(2)
           return true;
         };
         for (long long f = f_begin; f < f_end && ok; ++seg) {
@@ -269,41 +337,72 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const int n = (int)(seg_end - f);
           if (!mbar_wait(bar(Q_READY), seg & 1, s_abort)) { ok = false; break; }
           tc_fence_after();
-          if (!issue_qk(jt)) { ok = false; break; }
+          int issued = 0;                                  // score tiles of this segment already issued
           for (int i = 0; i < n; ++i) {
             const uint32_t j = jt + i;
-            if (i + 1 < n && !issue_qk(j + 1)) { ok = false; break; }
-            const uint32_t vs = j % kVStages, pb = j % kPBufs;
+            while (issued < n && issued <= i + NSB - 1) {  // look-ahead: keep NSB-1 score tiles in flight past tile i
+              if (!issue_qk(jt + issued)) { ok = false; break; }
+              ++issued;
+            }
+            if (!ok) break;
+            const uint32_t vs = j % kVStages, g = j & 1;
+            PROF_START
             if (i == 0 && seg > 0 && !mbar_wait(bar(O_FREE), (seg - 1) & 1, s_abort)) { ok = false; break; }
+            PROF_ADD(3)
             if (!mbar_wait(bar(V_FULL + vs), (j / kVStages) & 1, s_abort)) { ok = false; break; }
-            if (!mbar_wait(bar(P_FULL + pb), (j / kPBufs) & 1, s_abort)) { ok = false; break; }
+            PROF_ADD(4)
+            if (!mbar_wait(bar(P_FULL + g), (j >> 1) & 1, s_abort)) { ok = false; break; }
+            PROF_ADD(5)
             tc_fence_after();
-            const uint32_t v_base = smem_addr(sV + vs * kTileBytes), p_base = smem_addr(sP + pb * PBYTES);
+            const uint32_t v_base = smem_addr(sV + vs * kTileBytes), p_base = smem_addr(sP + g * PBYTES);
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
-              tc_mma(tmem_O, make_desc(v_base + kk * 2048, kBoxBytes, 1024, 2), make_desc(p_base + kk * 256, 128, 2048, 0),
-                     IDESC_PV, (i > 0 || kk > 0));
+              tc_mma(tmem_O + g * NRP, make_desc(v_base + kk * 2048, kBoxBytes, 1024, 2), make_desc(p_base + kk * 256, 128, 2048, 0),
+                     IDESC_PV, (i >= 2 || kk > 0));      // each group's accumulator starts afresh in every segment
             tc_commit(bar(V_EMPTY + vs));
-            tc_commit(bar(P_FREE + pb));
+            tc_commit(bar(P_FREE + g));
+            PROF_ADD(6)
           }
           if (!ok) break;
           tc_commit(bar(O_FULL));
           jt += n;
           f = seg_end;
         }
+        if (blockIdx.x == 0) PROF_DUMP(16)
       }
-    } else {
+    } else if (warp >= 4) {
       // =========================== softmax warps ===========================
+      asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+      // Two groups of four warps work on alternate tiles (group = tile parity), each with its own
+      // accumulator, reference m and row sums: two independent online-softmax streams whose
+      // partials the combine kernel merges.  A thread owns one key of its group's tile.
       const int q4 = warp & 3;                 // TMEM lane quarter this warp may access
-      const int wg = (warp - 2) >> 2;          // column half
+      const int g = (warp - 4) >> 2;           // softmax group
       const int t = q4 * 32 + lane;            // key within the tile == TMEM lane; channel d in the epilogue
-      const int st = tid - 64;                 // 0..255
-      const int col0 = wg * HALF;
+      const int st = tid - 128;                // 0..255
       const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
-      float m_loc[HALF], l_loc[HALF];
+      const int nch_valid = (a.rows + 15) >> 4; // chunks holding real query rows
+      float* m_s = s_m + g * 128;
+      float* fac_s = s_fac + g * 128;
+      int* newmax_s = s_newmax + g * 128;
+      float l_loc[NRP];
       uint32_t jt = 0;
       int seg = 0;
       bool ok = true;
+      PROF_DECL
+      auto group_sync = [&]() { asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory"); };
+      auto group_or = [&](bool pred) -> bool {
+        uint32_t out;
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.ne.u32 p, %1, 0;\n\t"
+            "bar.red.or.pred q, %2, 128, p;\n\t"
+            "selp.u32 %0, 1, 0, q;\n\t}"
+            : "=r"(out)
+            : "r"((uint32_t)pred), "r"(1 + g)
+            : "memory");
+        return out != 0;
+      };
       for (long long f = f_begin; f < f_end; ++seg) {
         const int item = (int)(f / Tt), tile0 = (int)(f - (long long)item * Tt);
         const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
@@ -314,146 +413,208 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * 128;
           for (int idx = st; idx < a.rows * 16; idx += kSoftmaxThreads) {
             const int row = idx >> 4, c = idx & 15;
-            const int r = row / a.G, g = row - r * a.G;
-            const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + g) * 128 + c * 8);
+            const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
+            const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * 128 + c * 8);
             *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val;
           }
           fence_proxy_async();
           mbar_arrive(bar(Q_READY));
         }
+        if (t < NRP) m_s[t] = kNegBig;
 #pragma unroll
-        for (int i = 0; i < HALF; ++i) { m_loc[i] = kNegBig; l_loc[i] = 0.f; }
+        for (int i = 0; i < NRP; ++i) l_loc[i] = 0.f;
+        group_sync();
 
         bool aborted = false;
-        for (int i = 0; i < n; ++i) {
-          const uint32_t j = jt + i, sb = j & 1, pb = j % kPBufs;
+        const int i_first = ((jt & 1) == (uint32_t)g) ? 0 : 1;      // this group's first tile in the segment
+        for (int i = i_first; i < n; i += 2) {
+          const uint32_t j = jt + i, sb = j % NSB;
           const int tile = tile0 + i;
-          const int key = tile * kTile + t;
+          const int rel = tile * kTile + t - a.n_ctx;                 // row r sees this key iff rel <= r
           const bool need_mask = (tile * kTile + kTile - 1 > a.n_ctx);
-          // A failed wait never leaves this loop on its own (the other softmax threads would be left
-          // at a named barrier): it clears `ok`, and the vote below takes all 256 threads out together.
-          ok &= mbar_wait(bar(S_FULL + sb), (j >> 1) & 1, s_abort);
+          const uint32_t s_addr = tmem_S + lane_addr + sb * NRP;
+          // A failed wait never leaves this loop on its own (the rest of the group would be left at a
+          // named barrier): it clears `ok`, and the vote below takes all 128 threads out together.
+          PROF_START
+          ok &= mbar_wait(bar(S_FULL + sb), (j / NSB) & 1, s_abort);
+          PROF_ADD(0)
           tc_fence_after();
-          float x[HALF];
-          auto load_scores = [&](bool subtract_m) {
-            uint32_t raw[NCH][8];
+          // ---- scores of this key against all rows: x = s * scale - m (log2 domain), masked ----
+          uint32_t xr[NCH][16];                       // TMEM loads land here and are converted in place
+          float xmax;
+          auto load_x = [&]() {
 #pragma unroll
-            for (int c = 0; c < NCH; ++c) tmem_ld8(tmem_S0 + lane_addr + sb * NRP + col0 + c * 8, raw[c]);
+            for (int c = 0; c < NCH; ++c)
+              if (c < nch_valid) tmem_ld16(s_addr + c * 16, xr[c]);
             tmem_wait_ld();
+            PROF_ADD(8)
+            float xm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            const float4* m4 = reinterpret_cast<const float4*>(m_s);
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
-              reg_fence8(raw[c]);
+              if (c < nch_valid) {
+                reg_fence16(xr[c]);
 #pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                const int idx = c * 8 + e;
-                float v = __uint_as_float(raw[c][e]) * a.scale_log2;
-                if (need_mask && key > a.n_ctx + (col0 + idx) / a.G) v = -INFINITY;
-                x[idx] = subtract_m ? v - m_loc[idx] : v;
+                for (int q = 0; q < 4; ++q) {
+                  const float4 mq = m4[c * 4 + q];
+                  const float v0 = fmaf(__uint_as_float(xr[c][4 * q + 0]), a.scale_log2, -mq.x);
+                  const float v1 = fmaf(__uint_as_float(xr[c][4 * q + 1]), a.scale_log2, -mq.y);
+                  const float v2 = fmaf(__uint_as_float(xr[c][4 * q + 2]), a.scale_log2, -mq.z);
+                  const float v3 = fmaf(__uint_as_float(xr[c][4 * q + 3]), a.scale_log2, -mq.w);
+                  xr[c][4 * q + 0] = __float_as_uint(v0);
+                  xr[c][4 * q + 1] = __float_as_uint(v1);
+                  xr[c][4 * q + 2] = __float_as_uint(v2);
+                  xr[c][4 * q + 3] = __float_as_uint(v3);
+                  xm[0] = fmaxf(xm[0], v0);
+                  xm[1] = fmaxf(xm[1], v1);
+                  xm[2] = fmaxf(xm[2], v2);
+                  xm[3] = fmaxf(xm[3], v3);
+                }
+              }
+            }
+            xmax = fmaxf(fmaxf(xm[0], xm[1]), fmaxf(xm[2], xm[3]));
+            if (need_mask) {                          // cold: only the last tile(s) of an item hold keys past a row's horizon
+              xmax = -INFINITY;
+#pragma unroll 1
+              for (int r = 0; r < 1; ++r) {           // (kept in its own block so that it stays out of the hot instruction stream)
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+#pragma unroll
+                  for (int e = 0; e < 16; ++e) {
+                    if (c < nch_valid) {
+                      if (rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16)) xr[c][e] = __float_as_uint(-INFINITY);
+                      xmax = fmaxf(xmax, __uint_as_float(xr[c][e]));
+                    }
+                  }
+                }
               }
             }
           };
-          load_scores(true);
-          bool exceed = false;
+          load_x();
+          PROF_ADD(1)
+          const bool slow = group_or((xmax > kRescaleThreshold) || !ok);
+          PROF_ADD(2)
+          if (slow) {
+            if (group_or(!ok)) { aborted = true; break; }              // uniform across the group
+            // ------- slow path: new per-row reference, rescale row sums and the accumulator -------
 #pragma unroll
-          for (int k = 0; k < HALF; ++k) exceed |= (x[k] > kRescaleThreshold);
-          if (softmax_bar_or(exceed || !ok)) {
-            if (softmax_bar_or(!ok)) { aborted = true; break; }        // uniform across the 256 threads
-            // ------- slow path: new per-row reference, rescale sums and accumulator -------
-            load_scores(false);
+            for (int c = 0; c < NCH; ++c) {
+              if (c < nch_valid) {
+                uint32_t raw[16];
+                tmem_ld16(s_addr + c * 16, raw);
+                tmem_wait_ld();
+                reg_fence16(raw);
 #pragma unroll
-            for (int k = 0; k < HALF; ++k) {
-              float v = x[k];
+                for (int e = 0; e < 16; ++e) {
+                  float v = __uint_as_float(raw[e]) * a.scale_log2;
+                  if (need_mask && rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16)) v = -INFINITY;
 #pragma unroll
-              for (int sh = 16; sh >= 1; sh >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, sh));
-              if (lane == 0) atomicMax(&s_newmax[col0 + k], f2ord(v));
+                  for (int sh = 16; sh >= 1; sh >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, sh));
+                  if (lane == 0) atomicMax(&newmax_s[c * 16 + e], f2ord(v));
+                }
+              }
             }
-            softmax_bar_sync();
-            float fac[HALF];
-#pragma unroll
-            for (int k = 0; k < HALF; ++k) {
-              const float mn = fmaxf(m_loc[k], ord2f(s_newmax[col0 + k]));
-              fac[k] = ex2(m_loc[k] - mn);             // 0 when the row had seen nothing, 1 when nothing changed
-              l_loc[k] *= fac[k];
-              m_loc[k] = mn;
+            group_sync();
+            if (t < NRP) {
+              const float mo = m_s[t], mn = fmaxf(mo, ord2f(newmax_s[t]));
+              fac_s[t] = ex2(mo - mn);                 // 0 when the row had seen nothing, 1 when nothing changed
+              m_s[t] = mn;
+              newmax_s[t] = f2ord(-INFINITY);
             }
-            if (i > 0) {
-              // the accumulator holds tiles < i: wait until the last of them has been added
-              ok &= mbar_wait(bar(P_FREE + ((j - 1) % kPBufs)), ((j - 1) / kPBufs) & 1, s_abort);
+            group_sync();
+#pragma unroll
+            for (int k = 0; k < NRP; ++k) l_loc[k] *= fac_s[k];
+            if (i >= 2) {
+              // the accumulator holds this group's earlier tiles: wait until the last of them has been added
+              ok &= mbar_wait(bar(P_FREE + g), ((j >> 1) - 1) & 1, s_abort);
               tc_fence_after();
 #pragma unroll
               for (int c = 0; c < NCH; ++c) {
-                uint32_t o[8];
-                tmem_ld8(tmem_O + lane_addr + col0 + c * 8, o);
+                uint32_t o[16];
+                tmem_ld16(tmem_O + lane_addr + g * NRP + c * 16, o);
                 tmem_wait_ld();
-                reg_fence8(o);
+                reg_fence16(o);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * fac[c * 8 + e]);
-                tmem_st8(tmem_O + lane_addr + col0 + c * 8, o);
+                for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * fac_s[c * 16 + e]);
+                tmem_st16(tmem_O + lane_addr + g * NRP + c * 16, o);
               }
               tmem_wait_st();
             }
-            softmax_bar_sync();                      // everyone has read s_newmax
-            if (st < NRP) s_newmax[st] = f2ord(-INFINITY);
-#pragma unroll
-            for (int k = 0; k < HALF; ++k) x[k] = x[k] - m_loc[k];
+            load_x();                                  // scores against the new reference
           }
+          PROF_ADD(3)
+          // the score buffer is no longer needed: let the issuer refill it
           tc_fence_before();
           mbar_arrive(bar(S_FREE + sb));
           // ---- probabilities, running sums, bf16 P in the MN-major core-matrix layout ----
-          if (j >= kPBufs) ok &= mbar_wait(bar(P_FREE + pb), ((j / kPBufs) - 1) & 1, s_abort);
-          unsigned char* pdst = sP + pb * PBYTES + (col0 >> 3) * 2048 + t * 16;
+          if (i >= 2) ok &= mbar_wait(bar(P_FREE + g), ((j >> 1) - 1) & 1, s_abort);
+          PROF_ADD(4)
+          unsigned char* pdst = sP + g * PBYTES + t * 16;
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
-            float p[8];
+            if (c < nch_valid) {
+              float p[16];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              p[e] = ex2(x[c * 8 + e]);
-              l_loc[c * 8 + e] += p[e];
+              for (int e = 0; e < 16; ++e) {
+                p[e] = ex2(__uint_as_float(xr[c][e]));
+                l_loc[c * 16 + e] += p[e];
+              }
+              *reinterpret_cast<uint4*>(pdst + (2 * c) * 2048) =
+                  make_uint4(pack2(p[0], p[1]), pack2(p[2], p[3]), pack2(p[4], p[5]), pack2(p[6], p[7]));
+              *reinterpret_cast<uint4*>(pdst + (2 * c + 1) * 2048) =
+                  make_uint4(pack2(p[8], p[9]), pack2(p[10], p[11]), pack2(p[12], p[13]), pack2(p[14], p[15]));
+            } else {
+              *reinterpret_cast<uint4*>(pdst + (2 * c) * 2048) = make_uint4(0, 0, 0, 0);
+              *reinterpret_cast<uint4*>(pdst + (2 * c + 1) * 2048) = make_uint4(0, 0, 0, 0);
             }
-            *reinterpret_cast<uint4*>(pdst + c * 2048) =
-                make_uint4(pack2(p[0], p[1]), pack2(p[2], p[3]), pack2(p[4], p[5]), pack2(p[6], p[7]));
           }
+          PROF_ADD(5)
           fence_proxy_async();
-          mbar_arrive(bar(P_FULL + pb));
+          mbar_arrive(bar(P_FULL + g));
+          PROF_ADD(6)
         }
-        if (aborted) break;
-        // ---- segment epilogue: partial O (fp32), and (m, l) per row ----
+        // both groups leave together: the exit vote is per group, so agree across groups here
+        if (softmax_bar_or(aborted)) break;
+        // ---- segment epilogue: this group's partial O (fp32), and (m, l) per row ----
         ok &= mbar_wait(bar(O_FULL), seg & 1, s_abort);
         tc_fence_after();
-        const long long slot = (long long)blockIdx.x * a.seg_max + (item - item_first);
+        const long long slot = ((long long)blockIdx.x * a.seg_max + (item - item_first)) * 2 + g;
         float* po = a.part_o + slot * NRP * 128;
+        const bool has_tiles = i_first < n;
+        if (has_tiles) {
 #pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-          uint32_t o[8];
-          tmem_ld8(tmem_O + lane_addr + col0 + c * 8, o);
-          tmem_wait_ld();
-          reg_fence8(o);
+          for (int c = 0; c < NCH; ++c) {
+            uint32_t o[16];
+            tmem_ld16(tmem_O + lane_addr + g * NRP + c * 16, o);
+            tmem_wait_ld();
+            reg_fence16(o);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) po[(long long)(col0 + c * 8 + e) * 128 + t] = __uint_as_float(o[e]);
+            for (int e = 0; e < 16; ++e) po[(long long)(c * 16 + e) * 128 + t] = __uint_as_float(o[e]);
+          }
         }
         tc_fence_before();
         mbar_arrive(bar(O_FREE));
 #pragma unroll
-        for (int k = 0; k < HALF; ++k) {
+        for (int k = 0; k < NRP; ++k) {
           float v = l_loc[k];
 #pragma unroll
           for (int sh = 16; sh >= 1; sh >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sh);
-          if (lane == 0) s_lsum[q4 * 128 + col0 + k] = v;
+          if (lane == 0) s_lsum[(g * 4 + q4) * 128 + k] = v;
         }
-        // m is identical in all threads of a column half; thread with t == 0 publishes it
-        if (t == 0) {
-#pragma unroll
-          for (int k = 0; k < HALF; ++k) a.part_ml[(slot * NRP + col0 + k) * 2] = m_loc[k];
+        group_sync();
+        if (t < NRP) {
+          const float* ls = s_lsum + g * 512;
+          const float l = ((ls[t] + ls[128 + t]) + ls[256 + t]) + ls[384 + t];
+          a.part_ml[(slot * NRP + t) * 2] = has_tiles ? m_s[t] : kNegBig;
+          a.part_ml[(slot * NRP + t) * 2 + 1] = has_tiles ? l : 0.f;
         }
-        softmax_bar_sync();
-        if (st < NRP) {
-          const float l = ((s_lsum[st] + s_lsum[128 + st]) + s_lsum[256 + st]) + s_lsum[384 + st];
-          a.part_ml[(slot * NRP + st) * 2 + 1] = l;
-        }
-        softmax_bar_sync();
+        group_sync();
+        PROF_ADD(7)
         jt += n;
         f = seg_end;
       }
+      if (blockIdx.x == 0 && st == 0) PROF_DUMP(28)
+      if (blockIdx.x == 0 && st == 255) PROF_DUMP(40)
     }
   }
 
@@ -470,7 +631,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   }
 }
 
-// Merge the segments of one (item, row): grid (rows, items), 128 threads (channel d).
+// Merge the partials of one (item, row): grid (rows, items), 128 threads (channel d).
 struct CombineArgs {
   const float *part_o, *part_ml;
   __nv_bfloat16* o;
@@ -490,17 +651,21 @@ __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs 
   float mstar = -INFINITY;
   for (long long c = c0; c < C && b(c) < hi; ++c) {
     if (b(c + 1) <= lo || b(c + 1) == b(c)) continue;
-    const long long slot = c * a.seg_max + (item - (int)(b(c) / a.tiles_per_item));
-    mstar = fmaxf(mstar, a.part_ml[(slot * a.nrp + row) * 2]);
+    const long long slot = (c * a.seg_max + (item - (int)(b(c) / a.tiles_per_item))) * 2;
+    for (int g = 0; g < 2; ++g)
+      if (a.part_ml[((slot + g) * a.nrp + row) * 2 + 1] > 0.f) mstar = fmaxf(mstar, a.part_ml[((slot + g) * a.nrp + row) * 2]);
   }
   float l = 0.f, acc = 0.f;
   for (long long c = c0; c < C && b(c) < hi; ++c) {
     if (b(c + 1) <= lo || b(c + 1) == b(c)) continue;
-    const long long slot = c * a.seg_max + (item - (int)(b(c) / a.tiles_per_item));
-    const float m = a.part_ml[(slot * a.nrp + row) * 2], ls = a.part_ml[(slot * a.nrp + row) * 2 + 1];
-    const float w = ex2(m - mstar);                     // 0 for a segment in which the row saw no key
-    l += ls * w;
-    acc += a.part_o[(slot * a.nrp + row) * 128 + d] * w;
+    const long long slot = (c * a.seg_max + (item - (int)(b(c) / a.tiles_per_item))) * 2;
+    for (int g = 0; g < 2; ++g) {
+      const float m = a.part_ml[((slot + g) * a.nrp + row) * 2], ls = a.part_ml[((slot + g) * a.nrp + row) * 2 + 1];
+      if (!(ls > 0.f)) continue;                        // a stream in which the row saw no key (or that had no tile)
+      const float w = ex2(m - mstar);
+      l += ls * w;
+      acc += a.part_o[((slot + g) * a.nrp + row) * 128 + d] * w;
+    }
   }
   const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
   const int r = row / a.G, g = row - r * a.G;
@@ -546,8 +711,8 @@ bool make_kv_map(CUtensorMap* map, const void* base, const pvlm_attn_params& p, 
 
 template <int NRP>
 constexpr int tc_smem_bytes() {
-  return 1024 /*alignment slack*/ + (kKStages + kVStages) * kTileBytes + 2 * NRP * 128 + p_bufs(NRP) * NRP * 256 + 128 * 4 +
-         4 * 128 * 4 + 24 * 8 + 64;
+  return 1024 /*alignment slack*/ + (kKStages + kVStages) * kTileBytes + 2 * NRP * 128 + 2 * NRP * 256 + 3 * 256 * 4 +
+         1024 * 4 + 32 * 8 + 64;
 }
 
 template <int NRP>
@@ -563,17 +728,22 @@ bool make_attn_tc_plan(const pvlm_attn_params& p, AttnTcPlan& plan) {
   if (p.D != 128 || p.Hkv <= 0 || p.Hq % p.Hkv != 0) return false;
   const int G = p.Hq / p.Hkv;
   const int rows = G * p.R;
-  if (rows > 128) return false;
+  if (rows > 96) return false;                   // wider groups stay on the mma.sync kernel
   plan.nrp = (rows + 15) / 16 * 16;
   plan.T = p.n_ctx + p.R;
   plan.tiles_per_item = ceil_div(plan.T, kTile);
   plan.total_tiles = (long long)plan.tiles_per_item * p.Hkv * p.n_layers;
   plan.n_cta = (int)(plan.total_tiles < kNumSMs ? plan.total_tiles : kNumSMs);
+  if (const char* e = getenv("PVLM_TC_CTAS")) {     // test hook: fewer CTAs => longer tile runs and more segments per CTA
+    const int v = atoi(e);
+    if (v >= 1 && v < plan.n_cta) plan.n_cta = v;
+  }
   const long long per_cta = (plan.total_tiles + plan.n_cta - 1) / plan.n_cta;
   plan.seg_max = (int)((per_cta + plan.tiles_per_item - 1) / plan.tiles_per_item) + 1;
   size_t off = 0;
-  plan.off_part_o = off;  off += align_up((size_t)plan.n_cta * plan.seg_max * plan.nrp * 128 * 4, 256);
-  plan.off_part_ml = off; off += align_up((size_t)plan.n_cta * plan.seg_max * plan.nrp * 2 * 4, 256);
+  // two partial slots (one per softmax group) per segment
+  plan.off_part_o = off;  off += align_up((size_t)plan.n_cta * plan.seg_max * 2 * plan.nrp * 128 * 4, 256);
+  plan.off_part_ml = off; off += align_up((size_t)plan.n_cta * plan.seg_max * 2 * plan.nrp * 2 * 4, 256);
   plan.off_status = off;  off += 256;
   plan.total = off;
   return true;
@@ -593,6 +763,7 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   const float scale = (p.softmax_scale == 0.f) ? 1.0f / sqrtf((float)p.D) : p.softmax_scale;
   a.scale_log2 = scale * kLog2e;
   a.tiles_per_item = plan.tiles_per_item; a.total_tiles = plan.total_tiles; a.seg_max = plan.seg_max; a.n_cta = plan.n_cta;
+  a.g_magic = (65536u + a.G - 1) / a.G;
   cudaMemsetAsync(a.status, 0, 4, s);
   switch (plan.nrp) {
     case 16: launch_tc<16>(mk, mv, a, s); break;
@@ -601,8 +772,6 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
     case 64: launch_tc<64>(mk, mv, a, s); break;
     case 80: launch_tc<80>(mk, mv, a, s); break;
     case 96: launch_tc<96>(mk, mv, a, s); break;
-    case 112: launch_tc<112>(mk, mv, a, s); break;
-    case 128: launch_tc<128>(mk, mv, a, s); break;
     default: return PVLM_ERR_UNSUPPORTED;
   }
   CombineArgs c;
