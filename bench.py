@@ -182,6 +182,13 @@ def run_ours(args):
                 q_tok=torch.empty((1, cfg.gamma), dtype=torch.float32, device=dev))
 
     pa = binding.attn_params(Q, K, V, cfg.n_ctx, O, lse, mass, mass_layers=w["mass_layers"] if L > 1 else None)
+    # events the library records right around the kernel that streams K and V (the dominant kernel)
+    k_ev = [torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)]
+    for e in k_ev:
+        e.record()                                  # forces creation of the underlying cudaEvent_t
+    torch.cuda.synchronize()
+    pa.prof_event_begin, pa.prof_event_end = k_ev[0].cuda_event, k_ev[1].cuda_event
+    main_kernel_ms = []
     pp = binding.prune_params(mass_cur, mass_ref, 0, cfg.m, cfg.k_keep, kept, None, K, V, dK, dV)
     pc = binding.accept_params(tl, dl, tok, u, 1.0, outs)
 
@@ -225,6 +232,9 @@ def run_ours(args):
     t0.record()
     for i in range(args.steps):
         device_step(marks[i])
+        if i % 8 == 7 or i == args.steps - 1:       # sample the in-library kernel events (needs a sync: every 8th step)
+            k_ev[1].synchronize()
+            main_kernel_ms.append(k_ev[0].elapsed_time(k_ev[1]))
     t1.record()
     barrier()
     total_ms = t0.elapsed_time(t1)
@@ -264,7 +274,9 @@ def run_ours(args):
     peak, peak_kind = measured_peaks()
     ms_per_step = total_ms / args.steps
     attn_avg_ms = sum(attn_ms) / len(attn_ms)
-    achieved = ab_attn / (attn_avg_ms * 1e-3) / 1e9
+    kern_ms = sum(main_kernel_ms) / len(main_kernel_ms)
+    ab_kernel = L * (2 * T * cfg.Hkv * cfg.D * 2 + R * cfg.Hq * cfg.D * 2)      # K and V once, Q once; partials excluded
+    achieved = ab_kernel / (kern_ms * 1e-3) / 1e9
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(tpath):
@@ -286,10 +298,11 @@ def run_ours(args):
         "stages_us": {"attention": attn_avg_ms * 1e3, "prune_select_gather": sum(prune_ms) / len(prune_ms) * 1e3,
                       "softmax_accept": sum(acc_ms) / len(acc_ms) * 1e3},
         "step_gbs": (ab_attn + ab_prune + ab_acc) / (ms_per_step * 1e-3) / 1e9,
-        "roofline": {"bound": "hbm", "kernel": "attn_kernel<128,0> (+combine, +mass pass on 2 layers)",
+        "roofline": {"bound": "hbm", "kernel": "attn_tc_kernel (one launch streams K and V of all layers)",
                      "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": traffic,
-                     "algorithmic_bytes_per_launch": ab_attn,
+                     "algorithmic_bytes_per_launch": ab_kernel, "kernel_us": kern_ms * 1e3,
+                     "attention_call_gbs": ab_attn / (attn_avg_ms * 1e-3) / 1e9,
                      "stage_gbs": {"prune_select_gather": ab_prune / (sum(prune_ms) / len(prune_ms) * 1e-3) / 1e9,
                                    "softmax_accept": ab_acc / (sum(acc_ms) / len(acc_ms) * 1e-3) / 1e9}},
         "paper_context": "paper reports only end-to-end speedups on 8x L40S (3.36x LLaVA-OV-72B, 2.42x Qwen2.5-VL-32B); no kernel-level number",

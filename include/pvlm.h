@@ -94,6 +94,8 @@ typedef struct {
   float softmax_scale;         /* 0 => 1/sqrt(D)                                               */
   void *workspace;
   size_t workspace_bytes;
+  void *prof_event_begin; /* optional cudaEvent_t pair (NULL = off): recorded on the stream right before   */
+  void *prof_event_end;   /* and right after the one kernel that streams K and V, for per-kernel timing   */
 } pvlm_attn_params;
 
 /* Host-only; needs no GPU.  Returns 0 if the parameters are unsupported. */

@@ -39,7 +39,8 @@ class AttnParams(C.Structure):
                 ("kv_token_stride", C.c_longlong), ("kv_head_stride", C.c_longlong),
                 ("mass_layer_stride", C.c_longlong),
                 ("softmax_scale", C.c_float),
-                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("prof_event_begin", C.c_void_p), ("prof_event_end", C.c_void_p)]
 
 
 class PruneParams(C.Structure):

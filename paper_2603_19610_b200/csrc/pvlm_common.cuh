@@ -30,6 +30,8 @@ struct AttnTcPlan {           // tensor-core (tcgen05) path, D = 128
 };
 bool make_attn_tc_plan(const pvlm_attn_params& p, AttnTcPlan& plan);
 pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& plan, char* ws, float* lse2, cudaStream_t s);
+// mass pass on the tensor-core path: needs lse2 of every row (log2 domain) and a [n_mass][Hkv][T_pad] scratch
+pvlm_status launch_attn_mass_tc(const pvlm_attn_params& p, const float* lse2, float* part_mass, int* status, cudaStream_t s);
 
 struct AttnPlan {
   bool use_tc;     // main pass on tcgen05; the mma.sync kernel still runs the mass pass

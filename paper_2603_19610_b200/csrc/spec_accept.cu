@@ -95,14 +95,26 @@ __global__ void __launch_bounds__(128) accept_scan_kernel(const AccArgs a) {
   const int b = blockIdx.x;
   const float c = a.inv_temp * kLog2e;
   __shared__ int s_reject[64];
-  for (int row = threadIdx.x; row < a.rows; row += blockDim.x) {
+  // one warp per logit row: lanes take chunk partials round-robin, then a fixed-order butterfly merge
+  for (int row = threadIdx.x >> 5; row < a.rows; row += blockDim.x >> 5) {
     const float2* st = a.stats + ((long long)b * a.rows + row) * a.n_stat_chunks;
-    float m = st[0].x, l = st[0].y;
-    for (int ch = 1; ch < a.n_stat_chunks; ++ch) merge_ml(m, l, st[ch].x, st[ch].y, c);
-    const double lse = (double)m * (double)a.inv_temp + log((double)l);
-    a.lse[(long long)b * a.rows + row] = lse;
-    if (row <= a.gamma) { if (a.lse_p) a.lse_p[(long long)b * (a.gamma + 1) + row] = (float)lse; }
-    else if (a.lse_q) a.lse_q[(long long)b * a.gamma + row - a.gamma - 1] = (float)lse;
+    const int lane = threadIdx.x & 31;
+    float m = -INFINITY, l = 0.f;
+    for (int ch = lane; ch < a.n_stat_chunks; ch += 32) {
+      const float2 v = st[ch];
+      merge_ml(m, l, v.x, v.y, c);
+    }
+#pragma unroll
+    for (int sh = 16; sh >= 1; sh >>= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m, sh), l2 = __shfl_xor_sync(0xffffffffu, l, sh);
+      merge_ml(m, l, m2, l2, c);
+    }
+    if (lane == 0) {
+      const double lse = (double)m * (double)a.inv_temp + log((double)l);
+      a.lse[(long long)b * a.rows + row] = lse;
+      if (row <= a.gamma) { if (a.lse_p) a.lse_p[(long long)b * (a.gamma + 1) + row] = (float)lse; }
+      else if (a.lse_q) a.lse_q[(long long)b * a.gamma + row - a.gamma - 1] = (float)lse;
+    }
   }
   __syncthreads();
   for (int t = threadIdx.x; t < a.gamma; t += blockDim.x) {
@@ -192,29 +204,71 @@ __global__ void __launch_bounds__(kSampThreads) resid_sums_kernel(const AccArgs 
 __global__ void __launch_bounds__(kSampThreads) resid_pick_kernel(const AccArgs a) {
   const int b = blockIdx.x;
   const int n = a.n_accept[b];
-  __shared__ int s_mode, s_chunk, s_fallback, s_pick;
+  __shared__ int s_chunk, s_fallback, s_pick;
   __shared__ double s_base, s_target;
   __shared__ double wsum[kSampThreads / 32];
   const double* cs = a.csum + (long long)b * a.n_samp_chunks * 2;
   const int* cl = a.clast + (long long)b * a.n_samp_chunks * 2;
-  if (threadIdx.x == 0) {
-    double zr = 0.0;
-    for (int ch = 0; ch < a.n_samp_chunks; ++ch) zr += cs[2 * ch];
-    const int mode = (zr > 0.0) ? 0 : 1;          // no residual weight at all => draw from p
-    double z = 0.0;
-    for (int ch = 0; ch < a.n_samp_chunks; ++ch) z += cs[2 * ch + mode];
-    const double target = (double)a.u[(long long)b * (a.gamma + 1) + a.gamma] * z;
-    double run = 0.0;
-    int pick = -1, last = -1;
-    for (int ch = 0; ch < a.n_samp_chunks; ++ch) {
-      last = max(last, cl[2 * ch + mode]);
-      if (pick < 0 && run + cs[2 * ch + mode] > target) { pick = ch; s_base = run; }
-      run += cs[2 * ch + mode];
+  // block-wide fp64 reductions / scan over the chunk sums (chunks in index order, 256 per round)
+  const int lane_ = threadIdx.x & 31, warp_ = threadIdx.x >> 5;
+  __shared__ double red[kSampThreads / 32];
+  __shared__ int s_last;
+  auto block_sum = [&](double v) -> double {
+    v = warp_sum_d(v);
+    __syncthreads();
+    if (lane_ == 0) red[warp_] = v;
+    __syncthreads();
+    double t = 0.0;
+    for (int k = 0; k < kSampThreads / 32; ++k) t += red[k];
+    return t;
+  };
+  double zr_part = 0.0, zp_part = 0.0;
+  int last_r = -1, last_p = -1;
+  for (int ch = threadIdx.x; ch < a.n_samp_chunks; ch += kSampThreads) {
+    zr_part += cs[2 * ch];
+    zp_part += cs[2 * ch + 1];
+    last_r = max(last_r, cl[2 * ch]);
+    last_p = max(last_p, cl[2 * ch + 1]);
+  }
+  const double zr = block_sum(zr_part);
+  const int mode = (zr > 0.0) ? 0 : 1;             // no residual weight at all => draw from p
+  const double z = mode == 0 ? zr : block_sum(zp_part);
+  const double target = (double)a.u[(long long)b * (a.gamma + 1) + a.gamma] * z;
+  if (threadIdx.x == 0) { s_chunk = 0x7fffffff; s_last = -1; s_pick = 0x7fffffff; }
+  __syncthreads();
+  atomicMax(&s_last, mode == 0 ? last_r : last_p);
+  double run_base = 0.0;
+  for (int c0 = 0; c0 < a.n_samp_chunks; c0 += kSampThreads) {
+    const int ch = c0 + threadIdx.x;
+    const double v = ch < a.n_samp_chunks ? cs[2 * ch + mode] : 0.0;
+    double incl = v;
+#pragma unroll
+    for (int sh = 1; sh < 32; sh <<= 1) {
+      const double t = __shfl_up_sync(0xffffffffu, incl, sh);
+      if (lane_ >= sh) incl += t;
     }
-    s_mode = mode; s_chunk = pick; s_fallback = last; s_target = target; s_pick = 0x7fffffff;
+    __syncthreads();
+    if (lane_ == 31) red[warp_] = incl;
+    __syncthreads();
+    double off = run_base;
+    for (int k = 0; k < warp_; ++k) off += red[k];
+    incl += off;
+    if (ch < a.n_samp_chunks && incl > target && incl - v <= target) {   // first crossing: unique
+      if (atomicMin(&s_chunk, ch) > ch) s_base = incl - v;
+    }
+    double tot = run_base;
+    for (int k = 0; k < kSampThreads / 32; ++k) tot += red[k];
+    run_base = tot;
+    __syncthreads();
+    if (s_chunk != 0x7fffffff) break;
+  }
+  if (threadIdx.x == 0) {
+    s_target = target;
+    s_fallback = s_last;
+    if (s_chunk == 0x7fffffff) s_chunk = -1;
   }
   __syncthreads();
-  const int mode = s_mode, chunk = s_chunk;
+  const int chunk = s_chunk;
   int* out = a.out_tokens + (long long)b * (a.gamma + 1) + n;
   if (chunk < 0) {                                 // rounding left no crossing: last token with weight
     if (threadIdx.x == 0) *out = s_fallback;

@@ -108,6 +108,113 @@ __global__ void __launch_bounds__(kSelThreads) uvprune_select_kernel(const SelAr
   }
 }
 
+// Block-wide exclusive prefix sum over 1024 threads; `total` receives the block sum.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int sh = 1; sh < 32; sh <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, sh);
+    if (lane >= sh) incl += t;
+  }
+  __syncthreads();                       // warp_sums may still be read from a previous call
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_sums[lane], wi = w;
+#pragma unroll
+    for (int sh = 1; sh < 32; sh <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, wi, sh);
+      if (lane >= sh) wi += t;
+    }
+    warp_sums[lane] = wi - w;            // exclusive offset of each warp
+    if (lane == 31) warp_sums[32] = wi;  // block total
+  }
+  __syncthreads();
+  total = warp_sums[32];
+  return warp_sums[warp] + incl - v;
+}
+
+// Register-resident variant for m <= ITEMS * 1024: each thread owns ITEMS consecutive scores, keys
+// never leave registers, and the ordered compaction needs two block scans in all.
+template <int ITEMS>
+__global__ void __launch_bounds__(kSelThreads) uvprune_select_reg_kernel(const SelArgs a) {
+  __shared__ unsigned int hist[256];
+  __shared__ unsigned int s_prefix, s_remaining;
+  __shared__ int wsum[33];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int base = tid * ITEMS;
+  const int nv = min(max(a.m - base, 0), ITEMS);
+  uint32_t key[ITEMS];
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    key[i] = 0u;
+    if (i < nv) {
+      const float s = a.ref ? __fsub_rn(a.cur[base + i], a.ref[base + i]) : a.cur[base + i];
+      if (a.score) a.score[base + i] = s;
+      key[i] = score_key(s);
+    }
+  }
+  if (a.k == 0) return;
+  if (tid == 0) { s_prefix = 0u; s_remaining = (unsigned)a.k; }
+  uint32_t mask = 0u;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (tid < 256) hist[tid] = 0u;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    const unsigned remaining = s_remaining;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i)
+      if (i < nv && (key[i] & mask) == prefix) atomicAdd(&hist[(key[i] >> shift) & 0xFFu], 1u);
+    __syncthreads();
+    // bins in descending digit order across threads 0..255: find the bin where the running count reaches `remaining`
+    unsigned v = 0, incl = 0;
+    if (tid < 256) {
+      v = hist[255 - tid];
+      incl = v;
+#pragma unroll
+      for (int sh = 1; sh < 32; sh <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, sh);
+        if (lane >= sh) incl += t;
+      }
+      if (lane == 31) wsum[warp] = (int)incl;
+    }
+    __syncthreads();
+    if (tid < 256) {
+      for (int w = 0; w < warp; ++w) incl += (unsigned)wsum[w];
+      const unsigned excl = incl - v;
+      if (excl < remaining && incl >= remaining) {
+        s_prefix = prefix | ((uint32_t)(255 - tid) << shift);
+        s_remaining = remaining - excl;
+      }
+    }
+    mask |= (0xFFu << shift);
+    __syncthreads();
+  }
+  const uint32_t tau = s_prefix;
+  const int take_eq = (int)s_remaining;
+  int n_eq = 0;
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) n_eq += (i < nv && key[i] == tau) ? 1 : 0;
+  int total;
+  const int eq_before = block_exclusive_scan(n_eq, wsum, total);
+  int n_sel = 0, e = eq_before;
+  uint32_t selbits = 0u;
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    if (i < nv) {
+      const bool eq = key[i] == tau;
+      const bool sel = key[i] > tau || (eq && e < take_eq);
+      e += eq ? 1 : 0;
+      if (sel) { selbits |= (1u << i); ++n_sel; }
+    }
+  }
+  int pos = block_exclusive_scan(n_sel, wsum, total);
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i)
+    if (selbits & (1u << i)) a.kept[pos++] = base + i;
+}
+
 struct GatherArgs {
   const int4 *src_k, *src_v;
   int4 *dst_k, *dst_v;
@@ -154,7 +261,10 @@ pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s) {
   sa.kept = p.kept_idx;
   sa.m = p.m;
   sa.k = p.k;
-  if (p.m > 0) uvprune_select_kernel<<<1, kSelThreads, 0, s>>>(sa);
+  if (p.m > 0) {
+    if (p.m <= 32 * kSelThreads) uvprune_select_reg_kernel<32><<<1, kSelThreads, 0, s>>>(sa);
+    else uvprune_select_kernel<<<1, kSelThreads, 0, s>>>(sa);
+  }
   if (p.src_k) {
     GatherArgs g;
     g.src_k = (const int4*)p.src_k;

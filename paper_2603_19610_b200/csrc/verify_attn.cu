@@ -361,7 +361,9 @@ pvlm_status launch_dw(const AttnArgs& a, const pvlm_attn_params& p, const AttnPl
   cudaFuncSetAttribute(attn_kernel<D, 0, MAXW>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0);
   cudaFuncSetAttribute(attn_kernel<D, 0, MAXW>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
   if (!plan.use_tc) {
+    if (p.prof_event_begin) cudaEventRecord((cudaEvent_t)p.prof_event_begin, s);
     attn_kernel<D, 0, MAXW><<<grid, threads, smem0, s>>>(a);
+    if (p.prof_event_end) cudaEventRecord((cudaEvent_t)p.prof_event_end, s);
     if (plan.splits > 1) attn_combine_kernel<D><<<dim3(plan.rows, p.Hkv, p.n_layers), D, 0, s>>>(a);
   }
   if (p.mass) {
@@ -446,6 +448,7 @@ pvlm_status launch_verify_attn(const pvlm_attn_params& p, const AttnPlan& plan, 
     const pvlm_status st = launch_verify_attn_tc(p, plan.tc, ws + plan.off_tc, a.lse2, s);
     if (st != PVLM_OK) return st;
     if (!p.mass) return PVLM_OK;
+    return launch_attn_mass_tc(p, a.lse2, a.part_mass, (int*)(ws + plan.off_tc + plan.tc.off_status), s);
   }
   return p.D == 64 ? launch_d<64>(a, p, plan, s) : launch_d<128>(a, p, plan, s);
 }

@@ -631,7 +631,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   }
 }
 
-// Merge the partials of one (item, row): grid (rows, items), 128 threads (channel d).
 struct CombineArgs {
   const float *part_o, *part_ml;
   __nv_bfloat16* o;
@@ -640,42 +639,276 @@ struct CombineArgs {
   long long total_tiles, q_ls;
 };
 
+// One block per (layer, KV head) item: thread 0 lists the partial slots of the item once, then the
+// 128 threads (channel d) walk the rows.
 __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs a) {
-  const int row = blockIdx.x, item = blockIdx.y, d = threadIdx.x;
-  const long long W = a.total_tiles, C = a.n_cta;
-  const long long lo = (long long)item * a.tiles_per_item, hi = lo + a.tiles_per_item;
-  auto b = [&](long long c) { return (W * c) / C; };
-  long long c0 = (lo * C) / W;
-  while (c0 + 1 < C && b(c0 + 1) <= lo) ++c0;
-  while (c0 > 0 && b(c0) > lo) --c0;
-  float mstar = -INFINITY;
-  for (long long c = c0; c < C && b(c) < hi; ++c) {
-    if (b(c + 1) <= lo || b(c + 1) == b(c)) continue;
-    const long long slot = (c * a.seg_max + (item - (int)(b(c) / a.tiles_per_item))) * 2;
-    for (int g = 0; g < 2; ++g)
-      if (a.part_ml[((slot + g) * a.nrp + row) * 2 + 1] > 0.f) mstar = fmaxf(mstar, a.part_ml[((slot + g) * a.nrp + row) * 2]);
+  const int item = blockIdx.x, d = threadIdx.x;
+  __shared__ long long s_slot[2 * kNumSMs + 4];          // at most every CTA contributes two partials
+  __shared__ int s_n;
+  if (d == 0) {
+    const long long W = a.total_tiles, C = a.n_cta;
+    const long long lo = (long long)item * a.tiles_per_item, hi = lo + a.tiles_per_item;
+    auto b = [&](long long c) { return (W * c) / C; };
+    long long c0 = (lo * C) / W;
+    while (c0 + 1 < C && b(c0 + 1) <= lo) ++c0;
+    while (c0 > 0 && b(c0) > lo) --c0;
+    int n = 0;
+    for (long long c = c0; c < C && b(c) < hi && n < 2 * kNumSMs; ++c) {
+      if (b(c + 1) <= lo || b(c + 1) == b(c)) continue;
+      const long long slot = (c * a.seg_max + (item - (int)(b(c) / a.tiles_per_item))) * 2;
+      s_slot[n++] = slot;
+      s_slot[n++] = slot + 1;
+    }
+    s_n = n;
   }
-  float l = 0.f, acc = 0.f;
-  for (long long c = c0; c < C && b(c) < hi; ++c) {
-    if (b(c + 1) <= lo || b(c + 1) == b(c)) continue;
-    const long long slot = (c * a.seg_max + (item - (int)(b(c) / a.tiles_per_item))) * 2;
-    for (int g = 0; g < 2; ++g) {
-      const float m = a.part_ml[((slot + g) * a.nrp + row) * 2], ls = a.part_ml[((slot + g) * a.nrp + row) * 2 + 1];
-      if (!(ls > 0.f)) continue;                        // a stream in which the row saw no key (or that had no tile)
-      const float w = ex2(m - mstar);
-      l += ls * w;
-      acc += a.part_o[((slot + g) * a.nrp + row) * 128 + d] * w;
+  __syncthreads();
+  const int n = s_n;
+  const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
+  for (int row = 0; row < a.rows; ++row) {
+    float mstar = -INFINITY;
+    for (int i = 0; i < n; ++i) {
+      const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
+      if (ml.y > 0.f) mstar = fmaxf(mstar, ml.x);
+    }
+    float l = 0.f, acc = 0.f;
+    for (int i = 0; i < n; ++i) {
+      const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
+      if (!(ml.y > 0.f)) continue;                      // a stream in which the row saw no key (or that had no tile)
+      const float w = ex2(ml.x - mstar);
+      l += ml.y * w;
+      acc += a.part_o[(s_slot[i] * a.nrp + row) * 128 + d] * w;
+    }
+    const int r = row / a.G, g = row - r * a.G;
+    a.o[(long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * 128 + d] = __float2bfloat16_rn(acc / l);
+    if (d == 0) {
+      const long long li = (long long)layer * a.Hq * a.R + (kvh * a.G + g) * a.R + r;
+      const float v2 = mstar + log2f(l);
+      a.lse2[li] = v2;
+      if (a.lse) a.lse[li] = v2 * kLn2;
     }
   }
-  const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
-  const int r = row / a.G, g = row - r * a.G;
-  a.o[(long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * 128 + d] = __float2bfloat16_rn(acc / l);
-  if (d == 0) {
-    const long long li = (long long)layer * a.Hq * a.R + (kvh * a.G + g) * a.R + r;
-    const float v2 = mstar + log2f(l);
-    a.lse2[li] = v2;
-    if (a.lse) a.lse[li] = v2 * kLn2;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Mass pass on the same machinery: S^T = K . Q^T only (no V, no P, no accumulator).  With the final
+// lse of every row known, a thread turns its key's scores into probabilities and adds them over the
+// query rows, which in this orientation is a thread-local sum: mass_part[kv head][key].
+// ---------------------------------------------------------------------------------------------
+constexpr int kMassKStages = 4;
+
+struct TcMassArgs {
+  const __nv_bfloat16* q;
+  const float* lse2;         // [n_layers][Hq][R], log2 domain
+  float* part_mass;          // [n_mass][Hkv][T_pad]
+  int* status;
+  int R, Hq, Hkv, G, n_ctx, T, T_pad, rows;
+  long long q_ls;
+  float scale_log2;
+  int tiles_per_item, n_cta;
+  long long total_tiles;
+  uint32_t g_magic;
+  int mass_listed;
+  int mass_layer[8];
+};
+
+template <int NRP>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a) {
+  constexpr int NCH = NRP / 16;
+  constexpr int QBOX = NRP * 128;
+  constexpr int NSB = (512 / NRP) >= 4 ? 4 : (512 / NRP);
+  constexpr uint32_t NEED = NSB * NRP;
+  constexpr uint32_t TMEM_COLS = NEED <= 32 ? 32 : NEED <= 64 ? 64 : NEED <= 128 ? 128 : NEED <= 256 ? 256 : 512;
+  constexpr uint32_t IDESC_QK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NRP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char* sK = smem;
+  unsigned char* sQ = sK + kMassKStages * kTileBytes;
+  float* s_lse = reinterpret_cast<float*>(sQ + 2 * QBOX);            // [128] lse2 per row (pad rows: +big => p = 0)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_lse + 128);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 24);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  enum { K_FULL = 0, K_EMPTY = 4, S_FULL = 8, S_FREE = 12, Q_READY = 16 };
+  auto bar = [&](int i) { return smem_addr(bars + i); };
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const long long W = a.total_tiles;
+  const long long f_begin = (W * blockIdx.x) / a.n_cta, f_end = (W * (blockIdx.x + 1)) / a.n_cta;
+  const int Tt = a.tiles_per_item;
+
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) {
+      mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1);
+      mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), kGroupThreads);
+    }
+    mbar_init(bar(Q_READY), kSoftmaxThreads);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(s_tmem)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  for (int i = tid; i < 2 * QBOX / 16; i += kThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+
+  if (f_end > f_begin) {
+    const uint32_t total = (uint32_t)(f_end - f_begin);
+    if (warp == 0) {
+      if (lane == 0) {
+        for (uint32_t j = 0; j < total; ++j) {
+          const long long f = f_begin + j;
+          const int item = (int)(f / Tt), tile = (int)(f - (long long)item * Tt);
+          const int zrow = item / a.Hkv, kvh = item - zrow * a.Hkv;
+          const int layer = a.mass_listed ? a.mass_layer[zrow] : zrow;
+          const uint32_t ks = j % kMassKStages;
+          if (j >= kMassKStages && !mbar_wait(bar(K_EMPTY + ks), ((j / kMassKStages) - 1) & 1, s_abort)) break;
+          mbar_expect_tx(bar(K_FULL + ks), kTileBytes);
+          tma_load_4d(smem_addr(sK + ks * kTileBytes), &tm_k, bar(K_FULL + ks), 0, kvh, tile * kTile, layer);
+          tma_load_4d(smem_addr(sK + ks * kTileBytes + kBoxBytes), &tm_k, bar(K_FULL + ks), 64, kvh, tile * kTile, layer);
+        }
+      }
+    } else if (warp == 1) {
+      if (lane == 0) {
+        const uint32_t q_base = smem_addr(sQ);
+        uint32_t jt = 0;
+        int seg = 0;
+        bool ok = true;
+        for (long long f = f_begin; f < f_end && ok; ++seg) {
+          const int item = (int)(f / Tt);
+          const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
+          const int n = (int)(seg_end - f);
+          if (!mbar_wait(bar(Q_READY), seg & 1, s_abort)) break;
+          tc_fence_after();
+          for (int i = 0; i < n; ++i) {
+            const uint32_t j = jt + i, ks = j % kMassKStages, sb = j % NSB;
+            if (!mbar_wait(bar(K_FULL + ks), (j / kMassKStages) & 1, s_abort)) { ok = false; break; }
+            if (j >= NSB && !mbar_wait(bar(S_FREE + sb), ((j / NSB) - 1) & 1, s_abort)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t k_base = smem_addr(sK + ks * kTileBytes);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+              const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32, qoff = (kk >> 2) * QBOX + (kk & 3) * 32;
+              tc_mma(tmem + sb * NRP, make_desc(k_base + off, 16, 1024, 2), make_desc(q_base + qoff, 16, 1024, 2), IDESC_QK, kk > 0);
+            }
+            tc_commit(bar(S_FULL + sb));
+            tc_commit(bar(K_EMPTY + ks));
+          }
+          jt += n;
+          f = seg_end;
+        }
+      }
+    } else if (warp >= 4) {
+      const int q4 = warp & 3, g = (warp - 4) >> 2;
+      const int t = q4 * 32 + lane, st = tid - 128;
+      const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
+      const int nch_valid = (a.rows + 15) >> 4;
+      uint32_t jt = 0;
+      int seg = 0;
+      bool ok = true;
+      for (long long f = f_begin; f < f_end; ++seg) {
+        const int item = (int)(f / Tt), tile0 = (int)(f - (long long)item * Tt);
+        const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
+        const int n = (int)(seg_end - f);
+        const int zrow = item / a.Hkv, kvh = item - zrow * a.Hkv;
+        const int layer = a.mass_listed ? a.mass_layer[zrow] : zrow;
+        {
+          const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * 128;
+          for (int idx = st; idx < a.rows * 16; idx += kSoftmaxThreads) {
+            const int row = idx >> 4, c = idx & 15;
+            const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
+            const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * 128 + c * 8);
+            *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val;
+          }
+          if (st < 128) {
+            float v = 1.0e30f;
+            if (st < a.rows) {
+              const int r = (int)(((uint32_t)st * a.g_magic) >> 16), gq = st - r * a.G;
+              v = a.lse2[((long long)layer * a.Hq + kvh * a.G + gq) * a.R + r];
+            }
+            s_lse[st] = v;
+          }
+          fence_proxy_async();
+          mbar_arrive(bar(Q_READY));
+        }
+        softmax_bar_or(false);                     // s_lse visible to both groups
+        const int i_first = ((jt & 1) == (uint32_t)g) ? 0 : 1;
+        float* out = a.part_mass + ((long long)zrow * a.Hkv + kvh) * a.T_pad;
+        for (int i = i_first; i < n; i += 2) {
+          const uint32_t j = jt + i, sb = j % NSB;
+          const int tile = tile0 + i;
+          const int key = tile * kTile + t;
+          const int rel = key - a.n_ctx;
+          const bool need_mask = (tile * kTile + kTile - 1 > a.n_ctx);
+          ok &= mbar_wait(bar(S_FULL + sb), (j / NSB) & 1, s_abort);
+          tc_fence_after();
+          const uint32_t s_addr = tmem + lane_addr + sb * NRP;
+          uint32_t xr[NCH][16];
+#pragma unroll
+          for (int c = 0; c < NCH; ++c)
+            if (c < nch_valid) tmem_ld16(s_addr + c * 16, xr[c]);
+          tmem_wait_ld();
+          tc_fence_before();
+          mbar_arrive(bar(S_FREE + sb));
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          const float4* l4 = reinterpret_cast<const float4*>(s_lse);
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) {
+            if (c < nch_valid) {
+              reg_fence16(xr[c]);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float4 lq = l4[c * 4 + q];
+                float x0 = fmaf(__uint_as_float(xr[c][4 * q + 0]), a.scale_log2, -lq.x);
+                float x1 = fmaf(__uint_as_float(xr[c][4 * q + 1]), a.scale_log2, -lq.y);
+                float x2 = fmaf(__uint_as_float(xr[c][4 * q + 2]), a.scale_log2, -lq.z);
+                float x3 = fmaf(__uint_as_float(xr[c][4 * q + 3]), a.scale_log2, -lq.w);
+                if (need_mask) {
+                  const int n0 = c * 16 + 4 * q;
+                  if (rel > (int)(((uint32_t)(n0 + 0) * a.g_magic) >> 16)) x0 = -INFINITY;
+                  if (rel > (int)(((uint32_t)(n0 + 1) * a.g_magic) >> 16)) x1 = -INFINITY;
+                  if (rel > (int)(((uint32_t)(n0 + 2) * a.g_magic) >> 16)) x2 = -INFINITY;
+                  if (rel > (int)(((uint32_t)(n0 + 3) * a.g_magic) >> 16)) x3 = -INFINITY;
+                }
+                acc[0] += ex2(x0);
+                acc[1] += ex2(x1);
+                acc[2] += ex2(x2);
+                acc[3] += ex2(x3);
+              }
+            }
+          }
+          if (key < a.T) out[key] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+        }
+        // all score MMAs of the segment have been consumed by one of the groups: Q may be replaced
+        if (softmax_bar_or(!ok)) break;
+        jt += n;
+        f = seg_end;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*s_abort) {
+    if (tid == 0) atomicExch(a.status, 1);
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+__global__ void mass_reduce_tc_kernel(const float* part, float* mass, int Hkv, int T, int T_pad, long long mass_ls) {
+  const int zrow = blockIdx.y;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= T) return;
+  float acc = 0.f;
+  for (int h = 0; h < Hkv; ++h) acc += part[((long long)zrow * Hkv + h) * T_pad + j];      // fixed order
+  mass[(long long)zrow * mass_ls + j] = acc;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -722,7 +955,47 @@ void launch_tc(const CUtensorMap& mk, const CUtensorMap& mv, const TcArgs& a, cu
   attn_tc_kernel<NRP><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
 }
 
+template <int NRP>
+void launch_tc_mass(const CUtensorMap& mk, const TcMassArgs& a, cudaStream_t s) {
+  constexpr int smem = 1024 + kMassKStages * kTileBytes + 2 * NRP * 128 + 128 * 4 + 24 * 8 + 64;
+  cudaFuncSetAttribute(attn_tc_mass_kernel<NRP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  attn_tc_mass_kernel<NRP><<<a.n_cta, kThreads, smem, s>>>(mk, a);
+}
+
 }  // namespace
+
+pvlm_status launch_attn_mass_tc(const pvlm_attn_params& p, const float* lse2, float* part_mass, int* status, cudaStream_t s) {
+  const int G = p.Hq / p.Hkv, rows = G * p.R, nrp = (rows + 15) / 16 * 16;
+  const int T = p.n_ctx + p.R;
+  CUtensorMap mk;
+  if (!make_kv_map(&mk, p.k, p, T)) return PVLM_ERR_UNSUPPORTED;
+  TcMassArgs a;
+  a.q = (const __nv_bfloat16*)p.q; a.lse2 = lse2; a.part_mass = part_mass; a.status = status;
+  a.R = p.R; a.Hq = p.Hq; a.Hkv = p.Hkv; a.G = G; a.n_ctx = p.n_ctx; a.T = T; a.T_pad = (int)align_up(T, kAttnBN); a.rows = rows;
+  a.q_ls = p.q_layer_stride;
+  const float scale = (p.softmax_scale == 0.f) ? 1.0f / sqrtf((float)p.D) : p.softmax_scale;
+  a.scale_log2 = scale * kLog2e;
+  a.mass_listed = p.mass_layers != nullptr;
+  const int n_mass = a.mass_listed ? p.n_mass_layers : p.n_layers;
+  for (int i = 0; i < 8; ++i) a.mass_layer[i] = (a.mass_listed && i < p.n_mass_layers) ? p.mass_layers[i] : 0;
+  a.tiles_per_item = ceil_div(T, kTile);
+  a.total_tiles = (long long)a.tiles_per_item * p.Hkv * n_mass;
+  a.n_cta = (int)(a.total_tiles < kNumSMs ? a.total_tiles : kNumSMs);
+  a.g_magic = (65536u + G - 1) / G;
+  switch (nrp) {
+    case 16: launch_tc_mass<16>(mk, a, s); break;
+    case 32: launch_tc_mass<32>(mk, a, s); break;
+    case 48: launch_tc_mass<48>(mk, a, s); break;
+    case 64: launch_tc_mass<64>(mk, a, s); break;
+    case 80: launch_tc_mass<80>(mk, a, s); break;
+    case 96: launch_tc_mass<96>(mk, a, s); break;
+    case 112: launch_tc_mass<112>(mk, a, s); break;
+    case 128: launch_tc_mass<128>(mk, a, s); break;
+    default: return PVLM_ERR_UNSUPPORTED;
+  }
+  mass_reduce_tc_kernel<<<dim3(ceil_div(T, 256), n_mass), 256, 0, s>>>(part_mass, p.mass, p.Hkv, T, a.T_pad, p.mass_layer_stride);
+  return check_launch();
+}
 
 bool make_attn_tc_plan(const pvlm_attn_params& p, AttnTcPlan& plan) {
   if (p.D != 128 || p.Hkv <= 0 || p.Hq % p.Hkv != 0) return false;
@@ -765,6 +1038,7 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   a.tiles_per_item = plan.tiles_per_item; a.total_tiles = plan.total_tiles; a.seg_max = plan.seg_max; a.n_cta = plan.n_cta;
   a.g_magic = (65536u + a.G - 1) / a.G;
   cudaMemsetAsync(a.status, 0, 4, s);
+  if (p.prof_event_begin) cudaEventRecord((cudaEvent_t)p.prof_event_begin, s);
   switch (plan.nrp) {
     case 16: launch_tc<16>(mk, mv, a, s); break;
     case 32: launch_tc<32>(mk, mv, a, s); break;
@@ -774,12 +1048,13 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
     case 96: launch_tc<96>(mk, mv, a, s); break;
     default: return PVLM_ERR_UNSUPPORTED;
   }
+  if (p.prof_event_end) cudaEventRecord((cudaEvent_t)p.prof_event_end, s);
   CombineArgs c;
   c.part_o = a.part_o; c.part_ml = a.part_ml; c.o = (__nv_bfloat16*)p.o; c.lse = p.lse; c.lse2 = lse2;
   c.R = p.R; c.Hq = p.Hq; c.Hkv = p.Hkv; c.G = a.G; c.rows = a.rows; c.nrp = plan.nrp;
   c.tiles_per_item = plan.tiles_per_item; c.seg_max = plan.seg_max; c.n_cta = plan.n_cta;
   c.total_tiles = plan.total_tiles; c.q_ls = p.q_layer_stride;
-  attn_tc_combine_kernel<<<dim3(a.rows, p.Hkv * p.n_layers), 128, 0, s>>>(c);
+  attn_tc_combine_kernel<<<p.Hkv * p.n_layers, 128, 0, s>>>(c);
   return check_launch();
 }
 
