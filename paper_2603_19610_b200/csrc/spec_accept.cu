@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(kStatThreads) row_stats_kernel(const AccArgs a
   }
 }
 
-__global__ void __launch_bounds__(128) accept_scan_kernel(const AccArgs a) {
+__global__ void __launch_bounds__(1024) accept_scan_kernel(const AccArgs a) {
   const int b = blockIdx.x;
   const float c = a.inv_temp * kLog2e;
   __shared__ int s_reject[64];
@@ -357,7 +357,7 @@ pvlm_status launch_spec_accept(const pvlm_accept_params& p, const AcceptPlan& pl
   a.clast = (int*)(ws + plan.off_clast);
   a.n_stat_chunks = plan.n_stat_chunks; a.n_samp_chunks = plan.n_samp_chunks;
   row_stats_kernel<<<dim3(plan.n_stat_chunks, plan.rows, p.batch), kStatThreads, 0, s>>>(a);
-  accept_scan_kernel<<<p.batch, 128, 0, s>>>(a);
+  accept_scan_kernel<<<p.batch, plan.rows > 32 ? 1024 : (plan.rows > 8 ? 512 : 128), 0, s>>>(a);
   resid_sums_kernel<<<dim3(plan.n_samp_chunks, p.batch), kSampThreads, 0, s>>>(a);
   resid_pick_kernel<<<p.batch, kSampThreads, 0, s>>>(a);
   if (p.probs_p || p.probs_q)

@@ -135,37 +135,52 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& 
   return warp_sums[warp] + incl - v;
 }
 
-// Register-resident variant for m <= ITEMS * 1024: each thread owns ITEMS consecutive scores, keys
-// never leave registers, and the ordered compaction needs two block scans in all.
+// Register-resident variant for m <= ITEMS * 1024.  Warp w owns the ITEMS*32 consecutive scores
+// starting at w*ITEMS*32; lane l holds elements w*ITEMS*32 + i*32 + l (coalesced loads), so index
+// order inside a warp is (i, lane) and ordered compaction needs only ballots plus two block scans.
 template <int ITEMS>
 __global__ void __launch_bounds__(kSelThreads) uvprune_select_reg_kernel(const SelArgs a) {
   __shared__ unsigned int hist[256];
+  __shared__ unsigned int hist_l[256 * 32];              // one histogram column per lane: bank = lane, so the
+                                                         // atomics of a warp never collide, whatever the digits
   __shared__ unsigned int s_prefix, s_remaining;
   __shared__ int wsum[33];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int base = tid * ITEMS;
-  const int nv = min(max(a.m - base, 0), ITEMS);
+  const int base = warp * (ITEMS * 32) + lane;
   uint32_t key[ITEMS];
+  uint32_t valid = 0u;
 #pragma unroll
   for (int i = 0; i < ITEMS; ++i) {
+    const int idx = base + i * 32;
     key[i] = 0u;
-    if (i < nv) {
-      const float s = a.ref ? __fsub_rn(a.cur[base + i], a.ref[base + i]) : a.cur[base + i];
-      if (a.score) a.score[base + i] = s;
+    if (idx < a.m) {
+      const float s = a.ref ? __fsub_rn(a.cur[idx], a.ref[idx]) : a.cur[idx];
+      if (a.score) a.score[idx] = s;
       key[i] = score_key(s);
+      valid |= 1u << i;
     }
   }
   if (a.k == 0) return;
+#ifdef PVLM_SEL_PROFILE
+  long long pt[6]; pt[0] = clock64();
+#endif
   if (tid == 0) { s_prefix = 0u; s_remaining = (unsigned)a.k; }
   uint32_t mask = 0u;
   for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0u;
+    for (int i = tid; i < 256 * 32; i += kSelThreads) hist_l[i] = 0u;
     __syncthreads();
     const uint32_t prefix = s_prefix;
     const unsigned remaining = s_remaining;
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i)
-      if (i < nv && (key[i] & mask) == prefix) atomicAdd(&hist[(key[i] >> shift) & 0xFFu], 1u);
+      if (((valid >> i) & 1u) && (key[i] & mask) == prefix) atomicAdd(&hist_l[(((key[i] >> shift) & 0xFFu) << 5) + lane], 1u);
+    __syncthreads();
+    if (tid < 256) {
+      unsigned t = 0;
+#pragma unroll 8
+      for (int j = 0; j < 32; ++j) t += hist_l[(tid << 5) + ((j + tid) & 31)];     // rotated: conflict-free
+      hist[tid] = t;
+    }
     __syncthreads();
     // bins in descending digit order across threads 0..255: find the bin where the running count reaches `remaining`
     unsigned v = 0, incl = 0;
@@ -193,26 +208,44 @@ __global__ void __launch_bounds__(kSelThreads) uvprune_select_reg_kernel(const S
   }
   const uint32_t tau = s_prefix;
   const int take_eq = (int)s_remaining;
-  int n_eq = 0;
+  const unsigned lt_mask = (1u << lane) - 1u;
+#ifdef PVLM_SEL_PROFILE
+  pt[1] = clock64();
+#endif
+  // equals per warp -> rank of every equal element in index order
+  int warp_eq = 0;
 #pragma unroll
-  for (int i = 0; i < ITEMS; ++i) n_eq += (i < nv && key[i] == tau) ? 1 : 0;
+  for (int i = 0; i < ITEMS; ++i) warp_eq += __popc(__ballot_sync(0xffffffffu, ((valid >> i) & 1u) && key[i] == tau));
   int total;
-  const int eq_before = block_exclusive_scan(n_eq, wsum, total);
-  int n_sel = 0, e = eq_before;
+  int eq_run = block_exclusive_scan(lane == 31 ? warp_eq : 0, wsum, total);   // lane 31 carries the warp's count
+  eq_run = __shfl_sync(0xffffffffu, eq_run, 31);                              // equals in all earlier warps
   uint32_t selbits = 0u;
+  int warp_sel = 0;
 #pragma unroll
   for (int i = 0; i < ITEMS; ++i) {
-    if (i < nv) {
-      const bool eq = key[i] == tau;
-      const bool sel = key[i] > tau || (eq && e < take_eq);
-      e += eq ? 1 : 0;
-      if (sel) { selbits |= (1u << i); ++n_sel; }
-    }
+    const bool v = (valid >> i) & 1u;
+    const bool eq = v && key[i] == tau;
+    const unsigned eq_b = __ballot_sync(0xffffffffu, eq);
+    const int rank = eq_run + __popc(eq_b & lt_mask);
+    const bool sel = v && (key[i] > tau || (eq && rank < take_eq));
+    eq_run += __popc(eq_b);
+    const unsigned sel_b = __ballot_sync(0xffffffffu, sel);
+    if (sel) selbits |= 1u << i;
+    warp_sel += __popc(sel_b);
   }
-  int pos = block_exclusive_scan(n_sel, wsum, total);
+  int pos = block_exclusive_scan(lane == 31 ? warp_sel : 0, wsum, total);
+  pos = __shfl_sync(0xffffffffu, pos, 31);                                    // selected in all earlier warps
 #pragma unroll
-  for (int i = 0; i < ITEMS; ++i)
-    if (selbits & (1u << i)) a.kept[pos++] = base + i;
+  for (int i = 0; i < ITEMS; ++i) {
+    const unsigned sel_b = __ballot_sync(0xffffffffu, (selbits >> i) & 1u);
+    if ((selbits >> i) & 1u) a.kept[pos + __popc(sel_b & lt_mask)] = base + i * 32;
+    pos += __popc(sel_b);
+  }
+#ifdef PVLM_SEL_PROFILE
+  pt[2] = clock64();
+  __syncthreads();
+  if (tid == 0) { a.kept[0] = (int)(pt[1] - pt[0]); a.kept[1] = (int)(pt[2] - pt[1]); a.kept[2] = (int)(pt[0] & 0x7fffffff); }
+#endif
 }
 
 struct GatherArgs {

@@ -639,13 +639,15 @@ struct CombineArgs {
   long long total_tiles, q_ls;
 };
 
-// One block per (layer, KV head) item: thread 0 lists the partial slots of the item once, then the
-// 128 threads (channel d) walk the rows.
+// Grid (items, kCombineSplit): thread 0 lists the partial slots of the item, then each warp merges
+// whole rows (a lane owns four channels), rows dealt round-robin over the grid's warps.
+constexpr int kCombineSplit = 8;
+
 __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs a) {
-  const int item = blockIdx.x, d = threadIdx.x;
+  const int item = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   __shared__ long long s_slot[2 * kNumSMs + 4];          // at most every CTA contributes two partials
   __shared__ int s_n;
-  if (d == 0) {
+  if (threadIdx.x == 0) {
     const long long W = a.total_tiles, C = a.n_cta;
     const long long lo = (long long)item * a.tiles_per_item, hi = lo + a.tiles_per_item;
     auto b = [&](long long c) { return (W * c) / C; };
@@ -664,23 +666,27 @@ __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs 
   __syncthreads();
   const int n = s_n;
   const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
-  for (int row = 0; row < a.rows; ++row) {
+  for (int row = blockIdx.y * 4 + warp; row < a.rows; row += 4 * kCombineSplit) {
     float mstar = -INFINITY;
     for (int i = 0; i < n; ++i) {
       const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
       if (ml.y > 0.f) mstar = fmaxf(mstar, ml.x);
     }
-    float l = 0.f, acc = 0.f;
+    float l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int i = 0; i < n; ++i) {
       const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
       if (!(ml.y > 0.f)) continue;                      // a stream in which the row saw no key (or that had no tile)
       const float w = ex2(ml.x - mstar);
       l += ml.y * w;
-      acc += a.part_o[(s_slot[i] * a.nrp + row) * 128 + d] * w;
+      const float4 o = *reinterpret_cast<const float4*>(a.part_o + (s_slot[i] * a.nrp + row) * 128 + lane * 4);
+      acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
     }
+    const float inv = 1.f / l;
     const int r = row / a.G, g = row - r * a.G;
-    a.o[(long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * 128 + d] = __float2bfloat16_rn(acc / l);
-    if (d == 0) {
+    __nv_bfloat16* dst = a.o + (long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * 128 + lane * 4;
+    *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(acc.x * inv, acc.y * inv), pack2(acc.z * inv, acc.w * inv));
+    if (lane == 0) {
       const long long li = (long long)layer * a.Hq * a.R + (kvh * a.G + g) * a.R + r;
       const float v2 = mstar + log2f(l);
       a.lse2[li] = v2;
@@ -1054,7 +1060,7 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   c.R = p.R; c.Hq = p.Hq; c.Hkv = p.Hkv; c.G = a.G; c.rows = a.rows; c.nrp = plan.nrp;
   c.tiles_per_item = plan.tiles_per_item; c.seg_max = plan.seg_max; c.n_cta = plan.n_cta;
   c.total_tiles = plan.total_tiles; c.q_ls = p.q_layer_stride;
-  attn_tc_combine_kernel<<<p.Hkv * p.n_layers, 128, 0, s>>>(c);
+  attn_tc_combine_kernel<<<dim3(p.Hkv * p.n_layers, kCombineSplit), 128, 0, s>>>(c);
   return check_launch();
 }
 
