@@ -43,7 +43,7 @@ def measured_peaks():
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
@@ -56,7 +56,9 @@ class ClockSampler:
         except OSError:
             self.p = None
 
-    def stop(self) -> dict:
+    def stop(self, t_begin: float = 0.0, t_end: float = 1e30) -> dict:
+        """Summarise the samples whose timestamp lies in [t_begin, t_end] (host wall clock)."""
+        import datetime
         if self.p is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.p.terminate()
@@ -66,23 +68,27 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         for line in self.f.read().strip().splitlines():
             parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 7:
+            if len(parts) < 8:
                 continue
             try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if ts < t_begin - 0.02 or ts > t_end + 0.02:
+                    continue
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+                pw.append(float(parts[3]))
             except ValueError:
                 continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[4:8]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         self.f.close()
         os.unlink(self.f.name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w": statistics.median(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
 # --------------------------------------------------------------------------------------
@@ -223,10 +229,11 @@ def run_ours(args):
         if marks is not None:
             marks[3].record()
 
+    sampler = ClockSampler(local_rank) if rank == 0 else None     # started early: nvidia-smi takes a while to deliver
     for _ in range(args.warmup):
         device_step()
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    wall_begin = time.time()
     marks = [[ev() for _ in range(4)] for _ in range(args.steps)]
     t0, t1 = ev(), ev()
     t0.record()
@@ -237,8 +244,9 @@ def run_ours(args):
             main_kernel_ms.append(k_ev[0].elapsed_time(k_ev[1]))
     t1.record()
     barrier()
+    wall_end = time.time()
     total_ms = t0.elapsed_time(t1)
-    clocks = sampler.stop() if sampler else None
+    clocks = sampler.stop(wall_begin, wall_end) if sampler else None
     attn_ms = [m[0].elapsed_time(m[1]) for m in marks]
     prune_ms = [m[1].elapsed_time(m[2]) for m in marks]
     acc_ms = [m[2].elapsed_time(m[3]) for m in marks]
@@ -398,7 +406,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2, help="workload index (2 = 32k-context, 64 layers: the metric's configuration)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")

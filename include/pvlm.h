@@ -88,8 +88,8 @@ typedef struct {
   int n_layers, R, Hq, Hkv, D, n_ctx;
   long long q_layer_stride;    /* elements */
   long long kv_layer_stride;   /* elements */
-  long long kv_token_stride;   /* elements, >= Hkv * kv_head_stride                            */
-  long long kv_head_stride;    /* elements, >= D                                               */
+  long long kv_token_stride;   /* elements, >= D (token-major [T][Hkv][D] and head-major      */
+  long long kv_head_stride;    /* elements, >= D  [Hkv][T][D] caches are both expressible)     */
   long long mass_layer_stride; /* elements, >= T                                               */
   float softmax_scale;         /* 0 => 1/sqrt(D)                                               */
   void *workspace;

@@ -61,9 +61,9 @@ pvlm_status pvlm_verify_attn(const pvlm_attn_params* p, void* stream) {
   if (!make_attn_plan(*p, plan)) return PVLM_ERR_UNSUPPORTED;
   if (!aligned(p->q, 16) || !aligned(p->k, 16) || !aligned(p->v, 16) || !aligned(p->o, 16)) return PVLM_ERR_INVALID_ARG;
   if (p->kv_head_stride < p->D || p->kv_head_stride % 8) return PVLM_ERR_INVALID_ARG;
-  if (p->kv_token_stride < (long long)p->Hkv * p->kv_head_stride || p->kv_token_stride % 8) return PVLM_ERR_INVALID_ARG;
+  if (p->kv_token_stride < p->D || p->kv_token_stride % 8) return PVLM_ERR_INVALID_ARG;   // token-major or head-major caches
   if (p->n_layers > 1) {
-    if (p->kv_layer_stride < (long long)plan.T * p->kv_token_stride || p->kv_layer_stride % 8) return PVLM_ERR_INVALID_ARG;
+    if (p->kv_layer_stride < (long long)plan.T * p->D || p->kv_layer_stride % 8) return PVLM_ERR_INVALID_ARG;
     if (p->q_layer_stride < (long long)p->R * p->Hq * p->D || p->q_layer_stride % 8) return PVLM_ERR_INVALID_ARG;
   }
   if (p->mass) {

@@ -11,7 +11,9 @@
 //                separate 2-deep shared-memory rings, completion on mbarriers.
 //   warp 1       MMA issuer (one thread): S^T = K . Q^T  (M = 128 keys, N = padded query rows,
 //                K = 128 channels) into one of up to four TMEM score buffers, then O^T += V^T . P^T
-//                (M = 128 channels, N = rows, K = 128 keys) into a TMEM output accumulator.
+//                (M = 128 channels, N = rows, K = 128 keys) into a TMEM output accumulator.  (Two
+//                separate issuer threads were tried: they let the two softmax groups fall into step,
+//                which loses the overlap between them.)
 //   warps 4..11  two softmax groups working on alternate tiles, each with its own accumulator,
 //                reference and row sums (two interleaved online-softmax streams).  A thread owns
 //                one key (TMEM lane) of its group's tile and all query-row columns, so exp2, the
@@ -57,6 +59,7 @@ struct TcArgs {
   int seg_max;               // partial slots per CTA
   int n_cta;
   uint32_t g_magic;          // ceil(2^16 / G): row / G == (row * g_magic) >> 16 for row < 128
+  int lookahead;             // score tiles the issuer keeps in flight past the tile whose PV it issues next
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -74,9 +77,19 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 // Bounded wait: false if the phase did not complete within the spin limit or another thread gave up.
+// A first non-blocking test_wait serves the common case of a phase that completed long ago (the
+// potentially-suspending try_wait costs a couple of hundred cycles even then).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  if (ok) return true;
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
@@ -170,11 +183,16 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
 #define PROF_START prof_t0 = clock64();
 #define PROF_ADD(i) { const long long now = clock64(); prof_acc[i] += now - prof_t0; prof_t0 = now; }
 #define PROF_DUMP(base) { for (int pi = 0; pi < 12; ++pi) a.status[(base) + pi] = (int)(prof_acc[pi] >> 4); }
+// event trace of tiles 400..407 of CTA 0: status[64 + ev * 8 + (tile - 400)] = clock
+#define TRACE_T0(ev, j) { if (t == 0) TRACE(ev, j) }
+#define TRACE(ev, j) { if (blockIdx.x == 0 && (j) >= 400u && (j) < 408u) a.status[64 + (ev) * 8 + ((j) - 400u)] = (int)(clock64() & 0x7fffffff); }
 #else
 #define PROF_DECL
 #define PROF_START
 #define PROF_ADD(i)
 #define PROF_DUMP(base) {}
+#define TRACE(ev, j)
+#define TRACE_T0(ev, j)
 #endif
 
 // ---------------------------------------------------------------------------------------------
@@ -255,9 +273,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // =========================== TMA producer ===========================
       if (lane == 0) {
         PROF_DECL
-        // K runs ahead of V by the MMA issuer's look-ahead, so the two rings advance separately:
-        // all K tiles first up to the ring depth, then alternate.
-        uint32_t jk = 0, jv = 0;
+        uint32_t jk = 0, jv = 0;                 // K and V rings advance separately: K leads by the score look-ahead
         const uint32_t total = (uint32_t)(f_end - f_begin);
         auto coords = [&](uint32_t j, int& kvh, int& tile, int& layer) {
           const long long f = f_begin + j;
@@ -266,9 +282,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           layer = item / a.Hkv;
           kvh = item - layer * a.Hkv;
         };
-        // The MMA issuer runs the score MMAs NSB-1 tiles ahead of the PV MMAs, so V(j) may only be
-        // waited for once K has been issued through tile j+NSB-1 (otherwise the issuer would wait for
-        // a K tile that this thread, blocked on a V slot, never sends).
+        // The MMA issuer runs the score MMAs `lookahead` tiles ahead of the PV MMAs, so V(j) may only be
+        // waited for once K has been issued through tile j+lookahead (otherwise the issuer would wait
+        // for a K tile that this thread, blocked on a V slot, never sends).
         while (jk < total || jv < total) {
           PROF_START
           // K tiles that must be on their way before PV(jv) can be issued; never past the end of
@@ -277,13 +293,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           if (jv < total) {
             const long long fv = f_begin + jv;
             const long long seg_end_j = min(f_end, (fv / Tt + 1) * (long long)Tt) - f_begin;
-            need_k = (uint32_t)min((long long)jv + NSB, seg_end_j);
+            need_k = (uint32_t)min((long long)jv + a.lookahead + 1, seg_end_j);
           }
           if (jk < total && jk < need_k) {
             const uint32_t ks = jk % kKStages;
             int kvh, tile, layer;
             coords(jk, kvh, tile, layer);
-            if (jk >= kKStages && !mbar_wait(bar(K_EMPTY + ks), ((jk / kKStages) - 1) & 1, s_abort)) break;
+            // slot ks was read by the score MMAs of tile jk-2: their completion is the S_FULL phase of that tile
+            if (jk >= kKStages && !mbar_wait(bar(S_FULL + (jk - kKStages) % NSB), ((jk - kKStages) / NSB) & 1, s_abort)) break;
             PROF_ADD(0)
             mbar_expect_tx(bar(K_FULL + ks), kTileBytes);
             tma_load_4d(smem_addr(sK + ks * kTileBytes), &tm_k, bar(K_FULL + ks), 0, kvh, tile * kTile, layer);
@@ -294,7 +311,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const uint32_t vs = jv % kVStages;
           int kvh, tile, layer;
           coords(jv, kvh, tile, layer);
-          if (jv >= kVStages && !mbar_wait(bar(V_EMPTY + vs), ((jv / kVStages) - 1) & 1, s_abort)) break;
+          // slot vs was read by the PV MMAs of tile jv-2: their completion is that group's P_FREE phase
+          if (jv >= kVStages && !mbar_wait(bar(P_FREE + ((jv - kVStages) & 1)), ((jv - kVStages) >> 1) & 1, s_abort)) break;
           PROF_ADD(1)
           mbar_expect_tx(bar(V_FULL + vs), kTileBytes);
           tma_load_4d(smem_addr(sV + vs * kTileBytes), &tm_v, bar(V_FULL + vs), 0, kvh, tile * kTile, layer);
@@ -306,12 +324,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       }
     } else if (warp == 1) {
       // =========================== MMA issuer ===========================
+      // One thread issues both MMA streams in order: score tiles run `lookahead` tiles ahead of the
+      // PV tiles, and the fixed interleave keeps the two softmax groups half a period apart.
       if (lane == 0) {
         const uint32_t q_base = smem_addr(sQ);
         bool ok = true;
         PROF_DECL
         uint32_t jt = 0;           // tiles issued by this CTA so far (ring phases run across segments)
         int seg = 0;
+#ifdef PVLM_TC_PROFILE
+        if (blockIdx.x == 0) {     // micro-timings of the synchronisation primitives (cycles per operation)
+          mbar_wait(bar(Q_READY), 0, s_abort);
+          long long c0 = clock64();
+          for (int r = 0; r < 64; ++r) mbar_wait(bar(Q_READY), 0, s_abort);
+          long long c1 = clock64();
+          for (int r = 0; r < 64; ++r) tc_fence_after();
+          long long c2 = clock64();
+          a.status[140] = (int)((c1 - c0) / 64);
+          a.status[141] = (int)((c2 - c1) / 64);
+        }
+#endif
         auto issue_qk = [&](uint32_t j) -> bool {
           const uint32_t ks = j % kKStages, sb = j % NSB;
           PROF_START
@@ -319,6 +351,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           PROF_ADD(0)
           if (j >= NSB && !mbar_wait(bar(S_FREE + sb), ((j / NSB) - 1) & 1, s_abort)) return false;
           PROF_ADD(1)
+          TRACE(0, j)
           tc_fence_after();
           const uint32_t k_base = smem_addr(sK + ks * kTileBytes);
 #pragma unroll
@@ -326,9 +359,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32, qoff = (kk >> 2) * QBOX + (kk & 3) * 32;
             tc_mma(tmem_S + sb * NRP, make_desc(k_base + off, 16, 1024, 2), make_desc(q_base + qoff, 16, 1024, 2), IDESC_QK, kk > 0);
           }
-          tc_commit(bar(S_FULL + sb));
-          tc_commit(bar(K_EMPTY + ks));
+          tc_commit(bar(S_FULL + sb));          // also frees the K slot (the K producer waits on this phase)
           PROF_ADD(2)
+          TRACE(1, j)
           return true;
         };
         for (long long f = f_begin; f < f_end && ok; ++seg) {
@@ -340,7 +373,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           int issued = 0;                                  // score tiles of this segment already issued
           for (int i = 0; i < n; ++i) {
             const uint32_t j = jt + i;
-            while (issued < n && issued <= i + NSB - 1) {  // look-ahead: keep NSB-1 score tiles in flight past tile i
+            while (issued < n && issued <= i + a.lookahead) {  // look-ahead: score tiles in flight past tile i
               if (!issue_qk(jt + issued)) { ok = false; break; }
               ++issued;
             }
@@ -353,15 +386,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             PROF_ADD(4)
             if (!mbar_wait(bar(P_FULL + g), (j >> 1) & 1, s_abort)) { ok = false; break; }
             PROF_ADD(5)
+            TRACE(2, j)
             tc_fence_after();
             const uint32_t v_base = smem_addr(sV + vs * kTileBytes), p_base = smem_addr(sP + g * PBYTES);
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
               tc_mma(tmem_O + g * NRP, make_desc(v_base + kk * 2048, kBoxBytes, 1024, 2), make_desc(p_base + kk * 256, 128, 2048, 0),
                      IDESC_PV, (i >= 2 || kk > 0));      // each group's accumulator starts afresh in every segment
-            tc_commit(bar(V_EMPTY + vs));
-            tc_commit(bar(P_FREE + g));
+            tc_commit(bar(P_FREE + g));          // also frees the V slot (the V producer waits on this phase)
             PROF_ADD(6)
+            TRACE(3, j)
           }
           if (!ok) break;
           tc_commit(bar(O_FULL));
@@ -438,6 +472,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           PROF_START
           ok &= mbar_wait(bar(S_FULL + sb), (j / NSB) & 1, s_abort);
           PROF_ADD(0)
+          TRACE_T0(4, j)
           tc_fence_after();
           // ---- scores of this key against all rows: x = s * scale - m (log2 domain), masked ----
           uint32_t xr[NCH][16];                       // TMEM loads land here and are converted in place
@@ -492,8 +527,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           };
           load_x();
           PROF_ADD(1)
+          TRACE_T0(5, j)
           const bool slow = group_or((xmax > kRescaleThreshold) || !ok);
           PROF_ADD(2)
+          TRACE_T0(6, j)
           if (slow) {
             if (group_or(!ok)) { aborted = true; break; }              // uniform across the group
             // ------- slow path: new per-row reference, rescale row sums and the accumulator -------
@@ -549,6 +586,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           // ---- probabilities, running sums, bf16 P in the MN-major core-matrix layout ----
           if (i >= 2) ok &= mbar_wait(bar(P_FREE + g), ((j >> 1) - 1) & 1, s_abort);
           PROF_ADD(4)
+          TRACE_T0(7, j)
           unsigned char* pdst = sP + g * PBYTES + t * 16;
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
@@ -572,6 +610,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           fence_proxy_async();
           mbar_arrive(bar(P_FULL + g));
           PROF_ADD(6)
+          TRACE_T0(8, j)
         }
         // both groups leave together: the exit vote is per group, so agree across groups here
         if (softmax_bar_or(aborted)) break;
@@ -1023,7 +1062,7 @@ bool make_attn_tc_plan(const pvlm_attn_params& p, AttnTcPlan& plan) {
   // two partial slots (one per softmax group) per segment
   plan.off_part_o = off;  off += align_up((size_t)plan.n_cta * plan.seg_max * 2 * plan.nrp * 128 * 4, 256);
   plan.off_part_ml = off; off += align_up((size_t)plan.n_cta * plan.seg_max * 2 * plan.nrp * 2 * 4, 256);
-  plan.off_status = off;  off += 256;
+  plan.off_status = off;  off += 8192;
   plan.total = off;
   return true;
 }
@@ -1043,6 +1082,14 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   a.scale_log2 = scale * kLog2e;
   a.tiles_per_item = plan.tiles_per_item; a.total_tiles = plan.total_tiles; a.seg_max = plan.seg_max; a.n_cta = plan.n_cta;
   a.g_magic = (65536u + a.G - 1) / a.G;
+  {
+    const int nsb = (512 - 2 * plan.nrp) / plan.nrp >= 4 ? 4 : (512 - 2 * plan.nrp) / plan.nrp;
+    a.lookahead = nsb - 1;
+    if (const char* e = getenv("PVLM_TC_LOOKAHEAD")) {      // tuning hook
+      const int v = atoi(e);
+      if (v >= 1 && v <= nsb - 1) a.lookahead = v;
+    }
+  }
   cudaMemsetAsync(a.status, 0, 4, s);
   if (p.prof_event_begin) cudaEventRecord((cudaEvent_t)p.prof_event_begin, s);
   switch (plan.nrp) {
