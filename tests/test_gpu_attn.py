@@ -136,3 +136,67 @@ def test_config3_and_4_geometry_full_context():
         cfg = wl.CONFIGS[cid]
         q, k, v = wl.attn_layer(cfg, 0)
         run_case(q, k, v, cfg.n_ctx)
+
+
+@pytest.mark.parametrize("ctas", [1, 3, 7])
+def test_tensor_core_path_long_tile_runs(ctas, monkeypatch):
+    """The tcgen05 kernel with few CTAs: long tile runs, several (layer, KV head) segments per CTA,
+    segments split between CTAs (the library reads PVLM_TC_CTAS when it plans a call)."""
+    monkeypatch.setenv("PVLM_TC_CTAS", str(ctas))
+    for (Hq, Hkv, D, n_ctx, R) in [(40, 8, 128, 2500, 13), (8, 2, 128, 1500, 5), (12, 4, 128, 700, 6)]:
+        qb, kb, vb = wl.make_qkv(Hq, Hkv, D, R, n_ctx + R, sink=True, seed=5 + n_ctx)
+        run_case(qb, kb, vb, n_ctx)
+
+
+def test_tensor_core_path_rescales_inside_long_runs(monkeypatch):
+    """Steeply growing scores inside one CTA's run: the lazy reference must be replaced many times,
+    rescaling the TMEM accumulator of each softmax group."""
+    monkeypatch.setenv("PVLM_TC_CTAS", "2")
+    Hq, Hkv, D, n_ctx, R = 8, 2, 128, 5000, 5
+    T = n_ctx + R
+    rq, rk, rv = (np.random.Generator(np.random.Philox(key=[17, i])) for i in range(3))
+    q, k, v = wl.make_qkv_f32(Hq, Hkv, D, R, T, False, rq, rk, rv)
+    k[:, :, D - 1] = (60.0 * np.arange(T) / T).astype(np.float32)[:, None]
+    run_case(wl.f32_to_bf16_bits(q), wl.f32_to_bf16_bits(k), wl.f32_to_bf16_bits(v), n_ctx)
+
+
+def test_mma_sync_path_still_matches(monkeypatch):
+    """PVLM_ATTN_IMPL=mma forces the mma.sync kernel for D = 128 as well (the second implementation)."""
+    monkeypatch.setenv("PVLM_ATTN_IMPL", "mma")
+    for (Hq, Hkv, D, n_ctx, R) in [(40, 8, 128, 2500, 13), (28, 4, 128, 1000, 9)]:
+        qb, kb, vb = wl.make_qkv(Hq, Hkv, D, R, n_ctx + R, sink=True, seed=9 + n_ctx)
+        run_case(qb, kb, vb, n_ctx)
+
+
+def test_head_major_cache_layout():
+    """K/V stored [Hkv][T][D] and passed through the strides."""
+    Hq, Hkv, D, n_ctx, R = 16, 4, 128, 900, 7
+    T = n_ctx + R
+    qb, kb, vb = wl.make_qkv(Hq, Hkv, D, R, T, sink=True, seed=44)
+    k = bf16_cuda(kb).permute(1, 0, 2).contiguous().permute(1, 0, 2)      # [T,Hkv,D] view of head-major storage
+    v = bf16_cuda(vb).permute(1, 0, 2).contiguous().permute(1, 0, 2)
+    assert k.stride(0) == D and k.stride(1) == T * D
+    o, lse, mass = binding.verify_attn(bf16_cuda(qb), k, v, n_ctx, want_mass=True, check=True)
+    torch.cuda.synchronize()
+    O, L, M = oracle_attn(qb, kb, vb, n_ctx)
+    assert_o_close(o, O)
+    assert_rel_close(mass.cpu().numpy(), M, what="mass")
+
+
+def test_timeout_status_is_reported_from_the_workspace_word():
+    """Failure reporting without making a GPU wait: the status word a bounded on-device wait would
+    set is poisoned from the host, and the health check must report PVLM_ERR_TIMEOUT."""
+    import ctypes as C
+    qb, kb, vb = wl.make_qkv(8, 2, 128, 3, 303, sink=False, seed=3)
+    q, k, v = bf16_cuda(qb), bf16_cuda(kb), bf16_cuda(vb)
+    o = torch.empty_like(q)
+    p = binding.attn_params(q, k, v, 300, o, None, None)
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert binding.lib().pvlm_verify_attn(C.byref(p), st) == 0
+    assert binding.lib().pvlm_verify_attn_check(C.byref(p), st) == 0
+    need = binding.lib().pvlm_verify_attn_workspace_bytes(C.byref(p))
+    ws = p._keep[6]
+    ws[need - 8192:need - 8188] = torch.tensor([1, 0, 0, 0], dtype=torch.uint8, device="cuda")   # the status word
+    assert binding.lib().pvlm_verify_attn_check(C.byref(p), st) == 6
+    assert binding.lib().pvlm_verify_attn(C.byref(p), st) == 0                                    # a new call clears it
+    assert binding.lib().pvlm_verify_attn_check(C.byref(p), st) == 0
