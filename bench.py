@@ -269,6 +269,10 @@ def run_ours(args):
     e2e_ms = e2e_t0.elapsed_time(e2e_t1)
     del e0
 
+    draft_report = None
+    if world == 1 and not args.no_draft_stream:
+        draft_report = draft_stream_leg(cfg, dev, torch, binding, wl, Q, K, V, O, lse, mass, w, pp, pc, args)
+
     if dist is not None:
         tt = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
@@ -315,11 +319,74 @@ def run_ours(args):
                                    "softmax_accept": ab_acc / (sum(acc_ms) / len(acc_ms) * 1e-3) / 1e9}},
         "paper_context": "paper reports only end-to-end speedups on 8x L40S (3.36x LLaVA-OV-72B, 2.42x Qwen2.5-VL-32B); no kernel-level number",
     }
+    if draft_report is not None:
+        out["draft_stream"] = draft_report
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, w)
     print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def draft_stream_leg(cfg, dev, torch, binding, wl, Q, K, V, O, lse, mass, w, pp, pc, args):
+    """Draft-decode stream beside the verify stream (the paper's parallel decoding stage): gamma sequential
+    decode steps of a 7B-shaped draft (28 layers, 28/4 heads, D = 128, one query row) over the compacted
+    cache on one stream, the verify -> prune -> accept step on another, SMs split between them."""
+    Ld, Hq_d, Hkv_d, D = 28, 28, 4, 128
+    draft_sms = args.draft_sms
+    S2 = cfg.T - cfg.m + cfg.k_keep
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    Kd = torch.randn((Ld, S2 + cfg.gamma, Hkv_d, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    Vd = torch.randn((Ld, S2 + cfg.gamma, Hkv_d, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    Qd = torch.randn((Ld, 1, Hq_d, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    Od = torch.empty_like(Qd)
+    sD = torch.cuda.Stream(device=dev)
+    L = cfg.n_layers
+    pa_split = binding.attn_params(Q, K, V, cfg.n_ctx, O, lse, mass, mass_layers=w["mass_layers"] if L > 1 else None,
+                                   max_ctas=148 - draft_sms)
+    with torch.cuda.stream(sD):                     # its own workspace: the two streams overlap on the GPU
+        pd = [binding.attn_params(Qd, Kd[:, :S2 + t + 1], Vd[:, :S2 + t + 1], S2 + t, Od, None, None, max_ctas=draft_sms)
+              for t in range(cfg.gamma)]
+
+    def verify():
+        binding.verify_step(pa_split, pp, pc, device=dev)
+
+    def draft():
+        with torch.cuda.stream(sD):
+            for p in pd:
+                binding.verify_step(p, None, None, device=dev)
+
+    def timed(fn_v, fn_d, reps):
+        ts = []
+        for _ in range(reps):
+            torch.cuda.synchronize()
+            e0 = torch.cuda.Event(enable_timing=True)
+            ev, ed = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            sD.wait_event(e0)
+            if fn_v:
+                fn_v()
+            ev.record()
+            if fn_d:
+                fn_d()
+            ed.record(sD)
+            torch.cuda.synchronize()
+            ts.append((e0.elapsed_time(ev) * 1e3, e0.elapsed_time(ed) * 1e3))
+        ts = ts[2:]
+        return (sum(t[0] for t in ts) / len(ts), sum(t[1] for t in ts) / len(ts))
+
+    reps = 12
+    v_alone, _ = timed(verify, None, reps)
+    _, d_alone = timed(None, draft, reps)
+    v_con, d_con = timed(verify, draft, reps)
+    draft_bytes = sum(Ld * 2 * (S2 + t + 1) * Hkv_d * D * 2 for t in range(cfg.gamma))
+    return {"sm_split": {"verify": 148 - draft_sms, "draft": draft_sms},
+            "draft_workload": f"{cfg.gamma} decode steps x {Ld} layers, {Hq_d}/{Hkv_d} heads, R=1, compacted cache {S2}+t rows "
+                              f"({draft_bytes / 1e9:.2f} GB of K/V per window)",
+            "verify_step_us_alone": v_alone, "draft_window_us_alone": d_alone,
+            "verify_step_us_concurrent": v_con, "draft_window_us_concurrent": d_con,
+            "both_us_concurrent": max(v_con, d_con), "both_us_serial": v_alone + d_alone}
 
 
 # --------------------------------------------------------------------------------------
@@ -411,6 +478,8 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="workload index (2 = 32k-context, 64 layers: the metric's configuration)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-draft-stream", action="store_true", help="skip the draft-stream concurrency leg")
+    ap.add_argument("--draft-sms", type=int, default=28, help="SMs left to the draft stream in the concurrency leg")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: truncate the config to this many layers (the JSON line says so)")
     args = ap.parse_args()

@@ -96,6 +96,9 @@ typedef struct {
   size_t workspace_bytes;
   void *prof_event_begin; /* optional cudaEvent_t pair (NULL = off): recorded on the stream right before   */
   void *prof_event_end;   /* and right after the one kernel that streams K and V, for per-kernel timing   */
+  int max_ctas;           /* 0 = one persistent CTA per SM.  A smaller value leaves SMs free for kernels   */
+                          /* of another stream (the draft model's decode steps run beside verification:   */
+                          /* paper Sec. 4.2, Stage II); the workspace query must see the same value.      */
 } pvlm_attn_params;
 
 /* Host-only; needs no GPU.  Returns 0 if the parameters are unsupported. */

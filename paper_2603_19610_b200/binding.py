@@ -40,7 +40,7 @@ class AttnParams(C.Structure):
                 ("mass_layer_stride", C.c_longlong),
                 ("softmax_scale", C.c_float),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("prof_event_begin", C.c_void_p), ("prof_event_end", C.c_void_p)]
+                ("prof_event_begin", C.c_void_p), ("prof_event_end", C.c_void_p), ("max_ctas", C.c_int)]
 
 
 class PruneParams(C.Structure):
@@ -138,7 +138,7 @@ def _stream(dev):
     return C.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
 
 
-def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None, mass_layers=None) -> AttnParams:
+def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None, mass_layers=None, max_ctas=0) -> AttnParams:
     """Fill an AttnParams from torch tensors: q/o [L,R,Hq,D] or [R,Hq,D]; k/v [L,T,Hkv,D] or [T,Hkv,D]."""
     if q.dim() == 3:
         q, k, v, o = q[None], k[None], v[None], o[None]
@@ -160,6 +160,7 @@ def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None, mass_la
     p.kv_layer_stride, p.kv_token_stride, p.kv_head_stride = k.stride(0), k.stride(1), k.stride(2)
     p.mass_layer_stride = mass.stride(0) if (mass is not None and mass.dim() == 2) else T
     p.softmax_scale = float(scale)
+    p.max_ctas = int(max_ctas)
     need = lib().pvlm_verify_attn_workspace_bytes(C.byref(p))
     ws = workspace if workspace is not None else _workspace(q.device, "attn", need)
     p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()
@@ -168,7 +169,7 @@ def attn_params(q, k, v, n_ctx, o, lse, mass, scale=0.0, workspace=None, mass_la
 
 
 def verify_attn(q, k, v, n_ctx: int, *, want_lse: bool = True, want_mass: bool = False, scale: float = 0.0,
-                out=None, workspace=None, mass_layers=None, check: bool = False):
+                out=None, workspace=None, mass_layers=None, check: bool = False, max_ctas: int = 0):
     """Window-verify GQA attention (see pvlm_verify_attn).  Returns (o, lse, mass).
 
     mass_layers (batched form only): list of layer indices whose mass is wanted;
@@ -182,7 +183,7 @@ def verify_attn(q, k, v, n_ctx: int, *, want_lse: bool = True, want_mass: bool =
     lse = torch.empty((L, Hq, R) if batched else (Hq, R), dtype=torch.float32, device=q.device) if want_lse else None
     n_mass = len(mass_layers) if mass_layers is not None else L
     mass = torch.empty((n_mass, T) if batched else (T,), dtype=torch.float32, device=q.device) if want_mass else None
-    p = attn_params(q, k, v, n_ctx, o, lse, mass, scale, workspace, mass_layers if want_mass else None)
+    p = attn_params(q, k, v, n_ctx, o, lse, mass, scale, workspace, mass_layers if want_mass else None, max_ctas)
     st = lib().pvlm_verify_attn(C.byref(p), _stream(q.device))
     if st != 0:
         raise PvlmError(st, "pvlm_verify_attn")

@@ -77,6 +77,7 @@ pvlm_status pvlm_verify_attn(const pvlm_attn_params* p, void* stream) {
     if (n_mass > 1 && p->mass_layer_stride < plan.T) return PVLM_ERR_INVALID_ARG;
   }
   if (p->n_layers > 65535 || p->Hkv > 65535) return PVLM_ERR_UNSUPPORTED;
+  if (p->max_ctas < 0) return PVLM_ERR_INVALID_ARG;
   const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, plan.total);
   if (w != PVLM_OK) return w;
   return launch_verify_attn(*p, plan, (cudaStream_t)stream);

@@ -1026,6 +1026,7 @@ pvlm_status launch_attn_mass_tc(const pvlm_attn_params& p, const float* lse2, fl
   a.tiles_per_item = ceil_div(T, kTile);
   a.total_tiles = (long long)a.tiles_per_item * p.Hkv * n_mass;
   a.n_cta = (int)(a.total_tiles < kNumSMs ? a.total_tiles : kNumSMs);
+  if (p.max_ctas > 0 && p.max_ctas < a.n_cta) a.n_cta = p.max_ctas;
   a.g_magic = (65536u + G - 1) / G;
   switch (nrp) {
     case 16: launch_tc_mass<16>(mk, a, s); break;
@@ -1052,6 +1053,7 @@ bool make_attn_tc_plan(const pvlm_attn_params& p, AttnTcPlan& plan) {
   plan.tiles_per_item = ceil_div(plan.T, kTile);
   plan.total_tiles = (long long)plan.tiles_per_item * p.Hkv * p.n_layers;
   plan.n_cta = (int)(plan.total_tiles < kNumSMs ? plan.total_tiles : kNumSMs);
+  if (p.max_ctas > 0 && p.max_ctas < plan.n_cta) plan.n_cta = p.max_ctas;
   if (const char* e = getenv("PVLM_TC_CTAS")) {     // test hook: fewer CTAs => longer tile runs and more segments per CTA
     const int v = atoi(e);
     if (v >= 1 && v < plan.n_cta) plan.n_cta = v;
