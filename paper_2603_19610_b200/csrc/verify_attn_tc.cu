@@ -124,6 +124,11 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
 }
+__device__ __forceinline__ void tmem_ld8_lo(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr));
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
@@ -200,10 +205,12 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
 // ---------------------------------------------------------------------------------------------
 __host__ __device__ constexpr int s_bufs(int nrp) { return (512 - 2 * nrp) / nrp >= 4 ? 4 : (512 - 2 * nrp) / nrp; }
 
-template <int NRP>
+// HT: the last 16-column chunk holds at most 8 real query rows, so only its first 8 columns are processed.
+template <int NRP, bool HT>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const TcArgs a) {
   constexpr int NCH = NRP / 16;            // 16-column chunks per thread
+  auto CW = [](int c) constexpr { return (HT && c == NRP / 16 - 1) ? 8 : 16; };   // processed columns of chunk c
   constexpr int QBOX = NRP * 128;          // bytes of one 64-channel box of Q
   constexpr int PBYTES = NRP * 256;        // one P buffer: NRP/8 row groups x 2048 B
   constexpr int NSB = s_bufs(NRP);         // score buffers in TMEM
@@ -257,7 +264,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // zero Q (its padding rows are never written again) and the slow-path scratch
-  for (int i = tid; i < 2 * QBOX / 16; i += kThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < (2 * QBOX + 2 * PBYTES) / 16; i += kThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);   // Q and both P buffers (contiguous)
   if (tid < 256) s_newmax[tid] = f2ord(-INFINITY);
   fence_proxy_async();
   tc_fence_before();
@@ -415,7 +422,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const int t = q4 * 32 + lane;            // key within the tile == TMEM lane; channel d in the epilogue
       const int st = tid - 128;                // 0..255
       const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
-      const int nch_valid = (a.rows + 15) >> 4; // chunks holding real query rows
       float* m_s = s_m + g * 128;
       float* fac_s = s_fac + g * 128;
       int* newmax_s = s_newmax + g * 128;
@@ -480,17 +486,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           auto load_x = [&]() {
 #pragma unroll
             for (int c = 0; c < NCH; ++c)
-              if (c < nch_valid) tmem_ld16(s_addr + c * 16, xr[c]);
+              if (CW(c) == 16) tmem_ld16(s_addr + c * 16, xr[c]); else tmem_ld8_lo(s_addr + c * 16, xr[c]);
             tmem_wait_ld();
             PROF_ADD(8)
             float xm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
             const float4* m4 = reinterpret_cast<const float4*>(m_s);
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
-              if (c < nch_valid) {
+              {
                 reg_fence16(xr[c]);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
+                for (int q = 0; q < CW(c) / 4; ++q) {
                   const float4 mq = m4[c * 4 + q];
                   const float v0 = fmaf(__uint_as_float(xr[c][4 * q + 0]), a.scale_log2, -mq.x);
                   const float v1 = fmaf(__uint_as_float(xr[c][4 * q + 1]), a.scale_log2, -mq.y);
@@ -515,8 +521,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
 #pragma unroll
-                  for (int e = 0; e < 16; ++e) {
-                    if (c < nch_valid) {
+                  for (int e = 0; e < CW(c); ++e) {
+                    {
                       if (rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16)) xr[c][e] = __float_as_uint(-INFINITY);
                       xmax = fmaxf(xmax, __uint_as_float(xr[c][e]));
                     }
@@ -536,13 +542,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             // ------- slow path: new per-row reference, rescale row sums and the accumulator -------
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
-              if (c < nch_valid) {
+              {
                 uint32_t raw[16];
                 tmem_ld16(s_addr + c * 16, raw);
                 tmem_wait_ld();
                 reg_fence16(raw);
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
+                for (int e = 0; e < CW(c); ++e) {
                   float v = __uint_as_float(raw[e]) * a.scale_log2;
                   if (need_mask && rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16)) v = -INFINITY;
 #pragma unroll
@@ -590,20 +596,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           unsigned char* pdst = sP + g * PBYTES + t * 16;
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
-            if (c < nch_valid) {
+            {
               float p[16];
 #pragma unroll
-              for (int e = 0; e < 16; ++e) {
+              for (int e = 0; e < CW(c); ++e) {
                 p[e] = ex2(__uint_as_float(xr[c][e]));
                 l_loc[c * 16 + e] += p[e];
               }
               *reinterpret_cast<uint4*>(pdst + (2 * c) * 2048) =
                   make_uint4(pack2(p[0], p[1]), pack2(p[2], p[3]), pack2(p[4], p[5]), pack2(p[6], p[7]));
-              *reinterpret_cast<uint4*>(pdst + (2 * c + 1) * 2048) =
-                  make_uint4(pack2(p[8], p[9]), pack2(p[10], p[11]), pack2(p[12], p[13]), pack2(p[14], p[15]));
-            } else {
-              *reinterpret_cast<uint4*>(pdst + (2 * c) * 2048) = make_uint4(0, 0, 0, 0);
-              *reinterpret_cast<uint4*>(pdst + (2 * c + 1) * 2048) = make_uint4(0, 0, 0, 0);
+              if (CW(c) == 16)                       // (the padding row group of a half chunk stays zero from start-up)
+                *reinterpret_cast<uint4*>(pdst + (2 * c + 1) * 2048) =
+                    make_uint4(pack2(p[8], p[9]), pack2(p[10], p[11]), pack2(p[12], p[13]), pack2(p[14], p[15]));
             }
           }
           PROF_ADD(5)
@@ -996,8 +1000,13 @@ constexpr int tc_smem_bytes() {
 template <int NRP>
 void launch_tc(const CUtensorMap& mk, const CUtensorMap& mv, const TcArgs& a, cudaStream_t s) {
   constexpr int smem = tc_smem_bytes<NRP>();
-  cudaFuncSetAttribute(attn_tc_kernel<NRP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  attn_tc_kernel<NRP><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
+  if (a.rows <= NRP - 8) {
+    cudaFuncSetAttribute(attn_tc_kernel<NRP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    attn_tc_kernel<NRP, true><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
+  } else {
+    cudaFuncSetAttribute(attn_tc_kernel<NRP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    attn_tc_kernel<NRP, false><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
+  }
 }
 
 template <int NRP>
