@@ -73,7 +73,8 @@ class StepParams(C.Structure):
                 ("h_target_logits", C.c_void_p), ("h_draft_logits", C.c_void_p),
                 ("h_draft_tokens", C.c_void_p), ("h_uniforms", C.c_void_p),
                 ("h_o", C.c_void_p), ("h_n_accept", C.c_void_p), ("h_out_tokens", C.c_void_p),
-                ("h_kept_idx", C.c_void_p)]
+                ("h_kept_idx", C.c_void_p),
+                ("copy_stream", C.c_void_p), ("event_a", C.c_void_p), ("event_b", C.c_void_p)]
 
 
 EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
@@ -298,14 +299,17 @@ def spec_accept(target_logits, draft_logits, draft_tokens, uniforms, temperature
 
 
 def verify_step(attn: AttnParams | None, prune: PruneParams | None, accept: AcceptParams | None, *,
-                host_in: dict | None = None, host_out: dict | None = None, device=None) -> StepParams:
+                host_in: dict | None = None, host_out: dict | None = None, device=None, overlap=None) -> StepParams:
     """One whole verify -> prune -> accept step through pvlm_verify_step.
 
     attn / prune / accept are parameter blocks built by attn_params / prune_params /
     accept_params (None skips the stage).  host_in maps h_q, h_k_window, h_v_window,
     h_target_logits, h_draft_logits, h_draft_tokens, h_uniforms to (pinned) CPU tensors
     copied to the device first; host_out maps h_o, h_n_accept, h_out_tokens, h_kept_idx to
-    CPU tensors filled at the end.  Asynchronous: synchronise the stream before reading."""
+    CPU tensors filled at the end.  overlap = (torch.cuda.Stream, torch.cuda.Event, torch.cuda.Event)
+    lets the library overlap the accept-input upload and the output download with compute (the
+    events must have been recorded once so that their handles exist).
+    Asynchronous: synchronise the stream before reading."""
     sp = StepParams()
     keep = []
     for name, blk in (("attn", attn), ("prune", prune), ("accept", accept)):
@@ -319,6 +323,10 @@ def verify_step(attn: AttnParams | None, prune: PruneParams | None, accept: Acce
                 assert not t.is_cuda and t.is_contiguous()
                 setattr(sp, k, C.c_void_p(t.data_ptr()))
                 keep.append(t)
+    if overlap is not None:
+        cs, ea, eb = overlap
+        sp.copy_stream, sp.event_a, sp.event_b = cs.cuda_stream, ea.cuda_event, eb.cuda_event
+        keep.append(overlap)
     dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
     st = lib().pvlm_verify_step(C.byref(sp), _stream(dev))
     if st != 0:

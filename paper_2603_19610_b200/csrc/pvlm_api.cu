@@ -158,11 +158,19 @@ pvlm_status pvlm_spec_accept(const pvlm_accept_params* p, void* stream) {
 pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
   if (!p) return PVLM_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
+  const bool overlap = p->copy_stream && p->event_a && p->event_b;
+  if (!overlap && (p->copy_stream || p->event_a || p->event_b)) return PVLM_ERR_INVALID_ARG;
+  cudaStream_t cs = overlap ? (cudaStream_t)p->copy_stream : s;      // stream of the overlappable copies
+  cudaEvent_t ea = (cudaEvent_t)p->event_a, eb = (cudaEvent_t)p->event_b;
   const pvlm_attn_params& a = p->attn;
   const pvlm_accept_params& c = p->accept;
   cudaError_t e = cudaSuccess;
   auto ok = [&]() { return e == cudaSuccess; };
   // ---- host -> device: this step's inputs ----
+  if (overlap) {                       // the copy stream starts after whatever is already queued on `stream`
+    e = cudaEventRecord(ea, s);
+    if (ok()) e = cudaStreamWaitEvent(cs, ea, 0);
+  }
   if (p->run_attn) {
     if (a.n_layers < 1 || a.R < 1 || a.Hq < 1 || a.Hkv < 1 || a.D < 1 || a.n_ctx < 0) return PVLM_ERR_INVALID_ARG;
     const size_t q_layer = (size_t)a.R * a.Hq * a.D * 2;
@@ -191,31 +199,42 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     }
     const size_t B = (size_t)c.batch;
     if (p->h_target_logits && ok())
-      e = cudaMemcpyAsync(const_cast<float*>(c.target_logits), p->h_target_logits, B * (c.gamma + 1) * c.V * 4, cudaMemcpyHostToDevice, s);
+      e = cudaMemcpyAsync(const_cast<float*>(c.target_logits), p->h_target_logits, B * (c.gamma + 1) * c.V * 4, cudaMemcpyHostToDevice, cs);
     if (p->h_draft_logits && ok())
-      e = cudaMemcpyAsync(const_cast<float*>(c.draft_logits), p->h_draft_logits, B * c.gamma * c.V * 4, cudaMemcpyHostToDevice, s);
+      e = cudaMemcpyAsync(const_cast<float*>(c.draft_logits), p->h_draft_logits, B * c.gamma * c.V * 4, cudaMemcpyHostToDevice, cs);
     if (p->h_draft_tokens && ok())
-      e = cudaMemcpyAsync(const_cast<int*>(c.draft_tokens), p->h_draft_tokens, B * c.gamma * 4, cudaMemcpyHostToDevice, s);
+      e = cudaMemcpyAsync(const_cast<int*>(c.draft_tokens), p->h_draft_tokens, B * c.gamma * 4, cudaMemcpyHostToDevice, cs);
     if (p->h_uniforms && ok())
-      e = cudaMemcpyAsync(const_cast<float*>(c.uniforms), p->h_uniforms, B * (c.gamma + 1) * 4, cudaMemcpyHostToDevice, s);
+      e = cudaMemcpyAsync(const_cast<float*>(c.uniforms), p->h_uniforms, B * (c.gamma + 1) * 4, cudaMemcpyHostToDevice, cs);
+    if (overlap && ok()) e = cudaEventRecord(ea, cs);           // accept inputs are on the device after this
   }
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   // ---- the three stages ----
   pvlm_status st;
   if (p->run_attn && (st = pvlm_verify_attn(&p->attn, stream)) != PVLM_OK) return st;
-  if (p->run_prune && (st = pvlm_uvprune_select_gather(&p->prune, stream)) != PVLM_OK) return st;
-  if (p->run_accept && (st = pvlm_spec_accept(&p->accept, stream)) != PVLM_OK) return st;
-  // ---- device -> host: this step's results ----
-  if (p->run_attn && p->h_o) {
+  if (p->run_attn && p->h_o) {                                   // o is final: its download may overlap the rest
     const size_t q_layer = (size_t)a.R * a.Hq * a.D * 2;
-    e = cudaMemcpy2DAsync(p->h_o, q_layer, a.o, (size_t)a.q_layer_stride * 2, q_layer, a.n_layers, cudaMemcpyDeviceToHost, s);
+    if (overlap) {
+      e = cudaEventRecord(eb, s);
+      if (ok()) e = cudaStreamWaitEvent(cs, eb, 0);
+    }
+    if (ok()) e = cudaMemcpy2DAsync(p->h_o, q_layer, a.o, (size_t)a.q_layer_stride * 2, q_layer, a.n_layers, cudaMemcpyDeviceToHost, cs);
+    if (overlap && ok()) e = cudaEventRecord(eb, cs);
+    if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   }
+  if (p->run_prune && (st = pvlm_uvprune_select_gather(&p->prune, stream)) != PVLM_OK) return st;
+  if (p->run_accept) {
+    if (overlap && (e = cudaStreamWaitEvent(s, ea, 0)) != cudaSuccess) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+    if ((st = pvlm_spec_accept(&p->accept, stream)) != PVLM_OK) return st;
+  }
+  // ---- device -> host: the rest of this step's results ----
   if (p->run_prune && p->h_kept_idx && p->prune.k > 0 && ok())
     e = cudaMemcpyAsync(p->h_kept_idx, p->prune.kept_idx, (size_t)p->prune.k * 4, cudaMemcpyDeviceToHost, s);
   if (p->run_accept && p->h_n_accept && ok())
     e = cudaMemcpyAsync(p->h_n_accept, c.n_accept, (size_t)c.batch * 4, cudaMemcpyDeviceToHost, s);
   if (p->run_accept && p->h_out_tokens && ok())
     e = cudaMemcpyAsync(p->h_out_tokens, c.out_tokens, (size_t)c.batch * (c.gamma + 1) * 4, cudaMemcpyDeviceToHost, s);
+  if (overlap && p->run_attn && p->h_o && ok()) e = cudaStreamWaitEvent(s, eb, 0);   // `stream` now also covers the o download
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   return PVLM_OK;
 }

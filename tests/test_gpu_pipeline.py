@@ -123,6 +123,18 @@ def test_verify_step_host_buffers_config0():
                  h_kept_idx=torch.zeros(cfg.k_keep, dtype=torch.int32).pin_memory())
     binding.verify_step(pa, pp, pc, host_in=h_in, host_out=h_out)
     torch.cuda.synchronize()
+    first = {k: v.clone() for k, v in h_out.items()}
+    # the same step with the accept-input upload and the o download overlapped on a copy stream
+    for host_t in h_out.values():
+        host_t.zero_()
+    tl2.zero_(); dl2.zero_(); q2.zero_(); o2.zero_()
+    cs, ea, eb = torch.cuda.Stream(), torch.cuda.Event(), torch.cuda.Event()
+    ea.record(); eb.record()
+    torch.cuda.synchronize()
+    binding.verify_step(pa, pp, pc, host_in=h_in, host_out=h_out, overlap=(cs, ea, eb))
+    torch.cuda.current_stream().synchronize()              # the caller's stream alone
+    for name in first:
+        assert torch.equal(first[name], h_out[name]), name
     assert torch.equal(h_out["h_o"], o_e.cpu())
     assert torch.equal(k2, k) and torch.equal(v2, v)                     # window rows landed in the cache
     assert torch.equal(h_out["h_kept_idx"], kept_e.cpu())
