@@ -2,6 +2,9 @@
 // lower-index tie break, ascending output) and the row gather that builds the
 // compacted draft cache.
 #include "pvlm_common.cuh"
+#include <cooperative_groups.h>
+#include <cstdlib>
+#include <cstring>
 #include <mutex>
 
 namespace pvlm {
@@ -248,6 +251,135 @@ __global__ void __launch_bounds__(kSelThreads) uvprune_select_reg_kernel(const S
 #endif
 }
 
+// Cluster variant: 8 CTAs (one thread-block cluster, 8 SMs) share the selection.  CTA r owns the
+// ITEMS*1024 consecutive scores starting at r*ITEMS*1024 (keys in registers, warp-coalesced as
+// above); per radix pass every CTA builds its own histogram, the cluster synchronises, and every CTA
+// adds up all eight histograms through distributed shared memory, so all CTAs derive the same
+// threshold without any global-memory round trip.  The ordered compaction needs one more exchange
+// (per-CTA counts of greater and of equal keys).  m <= 8 * 1024 * ITEMS.
+constexpr int kSelCluster = 8;
+
+template <int ITEMS>
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
+uvprune_select_cluster_kernel(const SelArgs a) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned rank = cluster.block_rank();
+  __shared__ unsigned int hist[256];                     // this CTA's histogram of the pass (read remotely)
+  __shared__ unsigned int hist_l[256 * 32];
+  __shared__ unsigned int s_prefix, s_remaining;
+  __shared__ int s_cnt[2];                               // (greater, equal) counts of this CTA (read remotely)
+  __shared__ int wsum[33];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int base = (int)rank * (ITEMS * kSelThreads) + warp * (ITEMS * 32) + lane;
+  uint32_t key[ITEMS];
+  uint32_t valid = 0u;
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const int idx = base + i * 32;
+    key[i] = 0u;
+    if (idx < a.m) {
+      const float s = a.ref ? __fsub_rn(a.cur[idx], a.ref[idx]) : a.cur[idx];
+      if (a.score) a.score[idx] = s;
+      key[i] = score_key(s);
+      valid |= 1u << i;
+    }
+  }
+  if (a.k == 0) return;                                  // uniform over the cluster: nobody reaches a cluster barrier
+  if (tid == 0) { s_prefix = 0u; s_remaining = (unsigned)a.k; }
+  uint32_t mask = 0u;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = tid; i < 256 * 32; i += kSelThreads) hist_l[i] = 0u;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    const unsigned remaining = s_remaining;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i)
+      if (((valid >> i) & 1u) && (key[i] & mask) == prefix) atomicAdd(&hist_l[(((key[i] >> shift) & 0xFFu) << 5) + lane], 1u);
+    __syncthreads();
+    if (tid < 256) {
+      unsigned t = 0;
+#pragma unroll 8
+      for (int j = 0; j < 32; ++j) t += hist_l[(tid << 5) + ((j + tid) & 31)];
+      hist[tid] = t;
+    }
+    cluster.sync();                                      // all eight histograms are complete
+    unsigned v = 0, incl = 0;
+    if (tid < 256) {
+#pragma unroll
+      for (int r = 0; r < kSelCluster; ++r) v += cluster.map_shared_rank(hist, r)[255 - tid];   // descending digit order
+      incl = v;
+#pragma unroll
+      for (int sh = 1; sh < 32; sh <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, sh);
+        if (lane >= sh) incl += t;
+      }
+      if (lane == 31) wsum[warp] = (int)incl;
+    }
+    __syncthreads();
+    if (tid < 256) {
+      for (int w = 0; w < warp; ++w) incl += (unsigned)wsum[w];
+      const unsigned excl = incl - v;
+      if (excl < remaining && incl >= remaining) {
+        s_prefix = prefix | ((uint32_t)(255 - tid) << shift);
+        s_remaining = remaining - excl;
+      }
+    }
+    mask |= (0xFFu << shift);
+    cluster.sync();                                      // remote reads of `hist` are done; s_prefix is visible
+  }
+  const uint32_t tau = s_prefix;
+  const int take_eq = (int)s_remaining;
+  const unsigned lt_mask = (1u << lane) - 1u;
+  int warp_eq = 0, warp_gt = 0;
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const bool vld = (valid >> i) & 1u;
+    warp_eq += __popc(__ballot_sync(0xffffffffu, vld && key[i] == tau));
+    warp_gt += __popc(__ballot_sync(0xffffffffu, vld && key[i] > tau));
+  }
+  int cta_eq, cta_gt;
+  int eq_run = block_exclusive_scan(lane == 31 ? warp_eq : 0, wsum, cta_eq);
+  eq_run = __shfl_sync(0xffffffffu, eq_run, 31);
+  block_exclusive_scan(lane == 31 ? warp_gt : 0, wsum, cta_gt);
+  if (tid == 0) { s_cnt[0] = cta_gt; s_cnt[1] = cta_eq; }
+  cluster.sync();
+  // counts of the CTAs before this one: equals before => how many of mine are kept; kept before => output offset
+  int eq_base = 0, sel_base = 0;
+  for (unsigned r = 0; r < rank; ++r) {
+    const int* c = cluster.map_shared_rank(s_cnt, r);
+    const int g = c[0], e = c[1];
+    const int kept_eq = min(max(take_eq - eq_base, 0), e);
+    sel_base += g + kept_eq;
+    eq_base += e;
+  }
+  cluster.sync();                                        // nobody leaves while its counts may still be read
+  eq_run += eq_base;
+  uint32_t selbits = 0u;
+  int warp_sel = 0;
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const bool vld = (valid >> i) & 1u;
+    const bool eq = vld && key[i] == tau;
+    const unsigned eq_b = __ballot_sync(0xffffffffu, eq);
+    const int rnk = eq_run + __popc(eq_b & lt_mask);
+    const bool sel = vld && (key[i] > tau || (eq && rnk < take_eq));
+    eq_run += __popc(eq_b);
+    const unsigned sel_b = __ballot_sync(0xffffffffu, sel);
+    if (sel) selbits |= 1u << i;
+    warp_sel += __popc(sel_b);
+  }
+  int total;
+  int pos = block_exclusive_scan(lane == 31 ? warp_sel : 0, wsum, total);
+  pos = __shfl_sync(0xffffffffu, pos, 31) + sel_base;
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const unsigned sel_b = __ballot_sync(0xffffffffu, (selbits >> i) & 1u);
+    if ((selbits >> i) & 1u) a.kept[pos + __popc(sel_b & lt_mask)] = base + i * 32;
+    pos += __popc(sel_b);
+  }
+}
+
 struct GatherArgs {
   const int4 *src_k, *src_v;
   int4 *dst_k, *dst_v;
@@ -295,7 +427,12 @@ pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s) {
   sa.m = p.m;
   sa.k = p.k;
   if (p.m > 0) {
-    if (p.m <= 32 * kSelThreads) uvprune_select_reg_kernel<32><<<1, kSelThreads, 0, s>>>(sa);
+    const char* impl = getenv("PVLM_SELECT_IMPL");       // "cta": single-CTA kernels only (second implementation for tests)
+    const bool one_cta = impl && strcmp(impl, "cta") == 0;
+    if (!one_cta && p.m <= kSelCluster * kSelThreads * 4) uvprune_select_cluster_kernel<4><<<kSelCluster, kSelThreads, 0, s>>>(sa);
+    else if (!one_cta && p.m <= kSelCluster * kSelThreads * 16) uvprune_select_cluster_kernel<16><<<kSelCluster, kSelThreads, 0, s>>>(sa);
+    else if (!one_cta && p.m <= kSelCluster * kSelThreads * 32) uvprune_select_cluster_kernel<32><<<kSelCluster, kSelThreads, 0, s>>>(sa);
+    else if (p.m <= 32 * kSelThreads) uvprune_select_reg_kernel<32><<<1, kSelThreads, 0, s>>>(sa);
     else uvprune_select_kernel<<<1, kSelThreads, 0, s>>>(sa);
   }
   if (p.src_k) {

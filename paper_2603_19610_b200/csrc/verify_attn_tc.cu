@@ -682,14 +682,15 @@ struct CombineArgs {
   long long total_tiles, q_ls;
 };
 
-// Grid (items, kCombineSplit): thread 0 lists the partial slots of the item, then each warp merges
-// whole rows (a lane owns four channels), rows dealt round-robin over the grid's warps.
-constexpr int kCombineSplit = 8;
-
+// Grid (items, rows): one block per query row.  Warp 0 lists the partial slots of the item; the four
+// warps then share the slots round-robin (a lane owns four channels) and their sums are merged in
+// fixed order through shared memory, so the result does not depend on timing.
 __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs a) {
   const int item = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   __shared__ long long s_slot[2 * kNumSMs + 4];          // at most every CTA contributes two partials
   __shared__ int s_n;
+  __shared__ float s_m[4], s_l[4];
+  __shared__ float4 s_acc[4][32];
   if (threadIdx.x == 0) {
     const long long W = a.total_tiles, C = a.n_cta;
     const long long lo = (long long)item * a.tiles_per_item, hi = lo + a.tiles_per_item;
@@ -708,33 +709,81 @@ __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs 
   }
   __syncthreads();
   const int n = s_n;
-  const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
-  for (int row = blockIdx.y * 4 + warp; row < a.rows; row += 4 * kCombineSplit) {
-    float mstar = -INFINITY;
-    for (int i = 0; i < n; ++i) {
-      const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
-      if (ml.y > 0.f) mstar = fmaxf(mstar, ml.x);
+  if (n <= 8) {
+    // few partials per item (long tile runs): a warp merges whole rows on its own, no block barriers
+    const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
+    for (int row = blockIdx.y * 4 + warp; row < a.rows; row += 4 * gridDim.y) {
+      float mstar = -INFINITY;
+      for (int i = 0; i < n; ++i) {
+        const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
+        if (ml.y > 0.f) mstar = fmaxf(mstar, ml.x);
+      }
+      float l = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int i = 0; i < n; ++i) {
+        const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
+        if (!(ml.y > 0.f)) continue;
+        const float w = ex2(ml.x - mstar);
+        l += ml.y * w;
+        const float4 o = *reinterpret_cast<const float4*>(a.part_o + (s_slot[i] * a.nrp + row) * 128 + lane * 4);
+        acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
+      }
+      const float inv = 1.f / l;
+      const int r = row / a.G, g = row - r * a.G;
+      __nv_bfloat16* dst = a.o + (long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * 128 + lane * 4;
+      *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(acc.x * inv, acc.y * inv), pack2(acc.z * inv, acc.w * inv));
+      if (lane == 0) {
+        const long long li = (long long)layer * a.Hq * a.R + (kvh * a.G + g) * a.R + r;
+        const float v2 = mstar + log2f(l);
+        a.lse2[li] = v2;
+        if (a.lse) a.lse[li] = v2 * kLn2;
+      }
     }
-    float l = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i = 0; i < n; ++i) {
-      const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
-      if (!(ml.y > 0.f)) continue;                      // a stream in which the row saw no key (or that had no tile)
-      const float w = ex2(ml.x - mstar);
-      l += ml.y * w;
-      const float4 o = *reinterpret_cast<const float4*>(a.part_o + (s_slot[i] * a.nrp + row) * 128 + lane * 4);
-      acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
-    }
-    const float inv = 1.f / l;
+    return;
+  }
+  for (int row = blockIdx.y; row < a.rows; row += gridDim.y) {
+  // reference = largest m among the partials that saw a key (every lane scans a strided share)
+  float mstar = -INFINITY;
+  for (int i = threadIdx.x; i < n; i += 128) {
+    const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
+    if (ml.y > 0.f) mstar = fmaxf(mstar, ml.x);
+  }
+#pragma unroll
+  for (int sh = 16; sh >= 1; sh >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, sh));
+  if (lane == 0) s_m[warp] = mstar;
+  __syncthreads();
+  mstar = fmaxf(fmaxf(s_m[0], s_m[1]), fmaxf(s_m[2], s_m[3]));
+  float l = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int i = warp; i < n; i += 4) {
+    const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
+    if (!(ml.y > 0.f)) continue;                        // a stream in which the row saw no key (or that had no tile)
+    const float w = ex2(ml.x - mstar);
+    l += ml.y * w;
+    const float4 o = *reinterpret_cast<const float4*>(a.part_o + (s_slot[i] * a.nrp + row) * 128 + lane * 4);
+    acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
+  }
+  s_acc[warp][lane] = acc;
+  if (lane == 0) s_l[warp] = l;
+  __syncthreads();
+  if (warp == 0) {
+    const float lt = ((s_l[0] + s_l[1]) + s_l[2]) + s_l[3];
+    float4 t = s_acc[0][lane];
+#pragma unroll
+    for (int w = 1; w < 4; ++w) { t.x += s_acc[w][lane].x; t.y += s_acc[w][lane].y; t.z += s_acc[w][lane].z; t.w += s_acc[w][lane].w; }
+    const float inv = 1.f / lt;
+    const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
     const int r = row / a.G, g = row - r * a.G;
     __nv_bfloat16* dst = a.o + (long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * 128 + lane * 4;
-    *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(acc.x * inv, acc.y * inv), pack2(acc.z * inv, acc.w * inv));
+    *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(t.x * inv, t.y * inv), pack2(t.z * inv, t.w * inv));
     if (lane == 0) {
       const long long li = (long long)layer * a.Hq * a.R + (kvh * a.G + g) * a.R + r;
-      const float v2 = mstar + log2f(l);
+      const float v2 = mstar + log2f(lt);
       a.lse2[li] = v2;
       if (a.lse) a.lse[li] = v2 * kLn2;
     }
+  }
+  __syncthreads();                                       // the shared staging arrays are reused by the next row
   }
 }
 
@@ -1118,7 +1167,12 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   c.R = p.R; c.Hq = p.Hq; c.Hkv = p.Hkv; c.G = a.G; c.rows = a.rows; c.nrp = plan.nrp;
   c.tiles_per_item = plan.tiles_per_item; c.seg_max = plan.seg_max; c.n_cta = plan.n_cta;
   c.total_tiles = plan.total_tiles; c.q_ls = p.q_layer_stride;
-  attn_tc_combine_kernel<<<dim3(p.Hkv * p.n_layers, kCombineSplit), 128, 0, s>>>(c);
+  {
+    const int items = p.Hkv * p.n_layers;
+    int rows_y = 2048 / items;                            // enough blocks to fill the GPU, not tens of thousands
+    rows_y = rows_y < 1 ? 1 : (rows_y > a.rows ? a.rows : rows_y);
+    attn_tc_combine_kernel<<<dim3(items, rows_y), 128, 0, s>>>(c);
+  }
   return check_launch();
 }
 

@@ -95,3 +95,27 @@ def test_select_from_oracle_masses_config0():
     cur, ref = m_cur.astype(np.float32), m_ref.astype(np.float32)
     kept, _ = gpu_select(cur, ref, 0, cfg.m, cfg.k_keep)
     np.testing.assert_array_equal(kept, select_topk(score_fp32(cur, ref, 0, cfg.m), cfg.k_keep))
+
+
+def test_single_cta_kernels_still_match(monkeypatch):
+    """PVLM_SELECT_IMPL=cta keeps the selection on the single-CTA kernels (register-resident up to
+    32,768 scores, global-memory keys above): the second implementation of the same selection."""
+    monkeypatch.setenv("PVLM_SELECT_IMPL", "cta")
+    rng = np.random.default_rng(77)
+    for m, k in [(30720, 3072), (131072, 6553), (5000, 4999)]:
+        cur = (np.round(rng.random(m) * 4096) / 4096).astype(np.float32)       # ties included
+        ref = rng.random(m).astype(np.float32)
+        kept, _ = gpu_select(cur, ref, 0, m, k, want_score=False)
+        np.testing.assert_array_equal(kept, select_topk(score_fp32(cur, ref, 0, m), k))
+        kept, _ = gpu_select(cur, None, 0, m, k, want_score=False)
+        np.testing.assert_array_equal(kept, select_topk(cur, k))
+
+
+def test_cluster_select_boundaries():
+    """Sizes around the per-CTA and per-variant boundaries of the 8-CTA cluster kernel, heavy ties."""
+    rng = np.random.default_rng(78)
+    for m in (4095, 4096, 4097, 32768, 32769, 131071, 131073, 262144):
+        cur = (np.round(rng.random(m) * 64) / 64).astype(np.float32)
+        for k in (1, m // 3, m - 1):
+            kept, _ = gpu_select(cur, None, 0, m, k, want_score=False)
+            np.testing.assert_array_equal(kept, select_topk(cur, k))
