@@ -13,5 +13,6 @@ Every function here is pinned by CPU tests to something other than itself
 tests); none is "parity unpinned".
 """
 from .attention import bf16_bits_to_f64, verify_attn  # noqa: F401
-from .uvprune import variation_score, select_topk, gather_rows  # noqa: F401
+from .uvprune import (variation_score, select_topk, gather_rows, cosine_similarity, similarity_sum,  # noqa: F401
+                      similarity_variation)
 from .accept import softmax64, spec_accept, window_size  # noqa: F401

@@ -20,6 +20,37 @@ from __future__ import annotations
 import numpy as np
 
 
+def cosine_similarity(hidden_bits, vis_start: int, m: int, text_start: int, n: int) -> np.ndarray:
+    """Eq. 1: S_ij = V_i . X_j / (|V_i| |X_j|) between the m visual rows and the n text rows of one
+    layer's token representations (bf16 bits [rows, d]).  Returns the full fp64 matrix [m, n].
+    A zero vector has similarity 0 with everything."""
+    b = np.ascontiguousarray(hidden_bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    h = b.view(np.float32).astype(np.float64)
+    V = h[vis_start:vis_start + m]
+    X = h[text_start:text_start + n]
+    nv = np.sqrt((V * V).sum(axis=1))
+    nx = np.sqrt((X * X).sum(axis=1))
+    S = V @ X.T
+    denom = nv[:, None] * nx[None, :]
+    return np.divide(S, denom, out=np.zeros_like(S), where=denom > 0)
+
+
+def similarity_sum(hidden_bits, vis_start: int, m: int, text_start: int, n: int) -> np.ndarray:
+    """sum_j S_ij: the per-layer relevance signal of visual token i (the inner sum of Eq. 2)."""
+    return cosine_similarity(hidden_bits, vis_start, m, text_start, n).sum(axis=1)
+
+
+def similarity_variation(hidden_layers, vis_start: int, m: int, text_start: int, n: int) -> np.ndarray:
+    """Eq. 2 as printed: sum over text tokens j and over layers l = 1..L of (S^l_ij - S^{l-1}_ij);
+    hidden_layers[0] is layer 0."""
+    S = [cosine_similarity(h, vis_start, m, text_start, n) for h in hidden_layers]
+    score = np.zeros(m)
+    for j in range(n):
+        for l in range(1, len(S)):
+            score += S[l][:, j] - S[l - 1][:, j]
+    return score
+
+
 def variation_score(mass_layers, vis_start: int, m: int) -> np.ndarray:
     """Eq. 2 as printed: sum over consecutive-layer differences, in fp64.
 

@@ -23,7 +23,7 @@ from numpy.random import Generator, Philox
 BASE_SEED = 260319000
 
 # random streams (one Philox key per (config, stream, layer))
-S_Q, S_K, S_V, S_REF, S_TLOGIT, S_DNOISE, S_DTOK, S_STEPU, S_STRUCT = range(9)
+S_Q, S_K, S_V, S_REF, S_TLOGIT, S_DNOISE, S_DTOK, S_STEPU, S_STRUCT, S_HIDDEN = range(10)
 
 
 @dataclass(frozen=True)
@@ -47,6 +47,7 @@ class Config:
     repeat_frac: float = 0.0  # share of frames drawn from one repeated pattern
     ref_layer: int = 0      # layer pair for the variation score (multi-layer)
     cur_layer: int = 0
+    d_model: int = 256      # width of the target's token representations (hidden-state criterion)
 
     @property
     def m(self) -> int:
@@ -78,14 +79,14 @@ class Config:
 
 
 CONFIGS = (
-    Config(0, "tiny", 4, 1, 64, 14, 64, 128, 4, 1024, 25, 1, False, 0.5),
-    Config(1, "qwen2.5-vl-7b-layer", 28, 4, 128, 64, 240, 1024, 8, 152064, 10, 1, True, 0.5),
+    Config(0, "tiny", 4, 1, 64, 14, 64, 128, 4, 1024, 25, 1, False, 0.5, d_model=256),
+    Config(1, "qwen2.5-vl-7b-layer", 28, 4, 128, 64, 240, 1024, 8, 152064, 10, 1, True, 0.5, d_model=3584),
     Config(2, "qwen2.5-vl-32b-64L", 40, 8, 128, 128, 240, 2048, 12, 152064, 10, 64, True, 0.5,
-           ref_layer=0, cur_layer=19),
+           ref_layer=0, cur_layer=19, d_model=5120),
     Config(3, "llava-ov-72b-80L", 64, 8, 128, 64, 196, 512, 10, 152064, 15, 80, True, 0.8,
-           ref_layer=0, cur_layer=19),
+           ref_layer=0, cur_layer=19, d_model=8192),
     Config(4, "long-video-stress", 40, 8, 128, 512, 256, 2048, 16, 152064, 5, 1, True, 0.5,
-           repeat_frac=0.3),
+           repeat_frac=0.3, d_model=5120),
 )
 
 
@@ -208,3 +209,29 @@ def kv_cache_layers(cfg: Config, n_layers: int, layer0: int = 0):
         ks.append(k)
         vs.append(v)
     return np.stack(ks), np.stack(vs)
+
+
+def hidden_layer(cfg: Config, layer: int, d_model: int | None = None, m: int | None = None, n: int | None = None):
+    """Token representations of one early target layer, bf16 bits [m + n, d]: visual rows then text
+    rows (the prefix order of Sec. 2.1).  Content is N(0,1) per layer; on top of it every row carries
+    a layer-invariant positional component beta(i) * p along a fixed direction p that the text rows
+    share (ramp towards the text boundary, spike on token 0), so that raw similarity favours the two
+    ends of the video and the layer-to-layer variation does not (Appendix E's argument)."""
+    d = d_model or cfg.d_model
+    m = cfg.m if m is None else m
+    n = cfg.n_text if n is None else n
+    rc = rng_for(cfg.cid, S_HIDDEN, layer + 1)
+    rp = rng_for(cfg.cid, S_HIDDEN, 0)                    # positional direction: the same in every layer
+    h = rc.standard_normal((m + n, d), dtype=np.float32)
+    p = rp.standard_normal(d, dtype=np.float32)
+    p *= np.float32(np.sqrt(d) / np.linalg.norm(p))
+    beta = np.zeros(m + n, dtype=np.float32)
+    beta[:m] = 0.6 * np.arange(m, dtype=np.float32) / max(m - 1, 1)
+    beta[0] += 1.0
+    beta[m:] = 0.8
+    h += beta[:, None] * p[None, :]
+    # a layer-dependent "semantic" gain for a seeded subset of visual tokens: these gain alignment with the text
+    sem = rng_for(cfg.cid, S_HIDDEN, 0).choice(m, size=max(1, m // 10), replace=False)
+    t_dir = h[m:].mean(axis=0)
+    h[sem] += np.float32(0.03 * layer) * t_dir[None, :]
+    return f32_to_bf16_bits(h)

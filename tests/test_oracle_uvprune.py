@@ -91,3 +91,72 @@ def test_variation_reduces_positional_concentration():
     share_var = (var >= last_q).mean()
     assert share_raw > 0.5
     assert share_var < share_raw - 0.15
+
+
+def _hidden(m, n, d, seed):
+    rng = np.random.default_rng(seed)
+    return wl.f32_to_bf16_bits(rng.standard_normal((m + n, d)).astype(np.float32))
+
+
+def test_cosine_brute_force_and_bounds():
+    """Eq. 1 against scalar loops; |S_ij| <= 1; scaling a row leaves its cosines unchanged."""
+    import math
+    from oracle.attention import bf16_bits_to_f64
+    from oracle.uvprune import cosine_similarity, similarity_sum
+    m, n, d = 7, 5, 16
+    hb = _hidden(m, n, d, 1)
+    S = cosine_similarity(hb, 0, m, m, n)
+    h = bf16_bits_to_f64(hb)
+    for i in range(m):
+        for j in range(n):
+            dot = sum(float(h[i, c]) * float(h[m + j, c]) for c in range(d))
+            ni = math.sqrt(sum(float(h[i, c]) ** 2 for c in range(d)))
+            nj = math.sqrt(sum(float(h[m + j, c]) ** 2 for c in range(d)))
+            assert abs(S[i, j] - dot / (ni * nj)) < 1e-12
+    assert np.abs(S).max() <= 1 + 1e-12
+    h2 = bf16_bits_to_f64(hb).astype(np.float32)
+    h2[2] *= 4.0                                             # exact in bf16
+    h2[m + 1] *= 0.5
+    S2 = cosine_similarity(wl.f32_to_bf16_bits(h2), 0, m, m, n)
+    np.testing.assert_allclose(S2, S, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(similarity_sum(hb, 0, m, m, n), S.sum(axis=1), rtol=1e-13)
+    # identical rows => cosine 1; opposite => -1; zero row => 0
+    h3 = h2.copy()
+    h3[0] = h3[m]
+    h3[1] = -h3[m]
+    h3[3] = 0.0
+    S3 = cosine_similarity(wl.f32_to_bf16_bits(h3), 0, m, m, n)
+    assert abs(S3[0, 0] - 1) < 1e-12 and abs(S3[1, 0] + 1) < 1e-12 and (S3[3] == 0).all()
+    # library routine: sklearn / scipy cosine distance
+    from scipy.spatial.distance import cdist
+    np.testing.assert_allclose(S, 1.0 - cdist(h[:m], h[m:], metric="cosine"), atol=1e-12)
+
+
+def test_similarity_variation_telescopes_to_end_layers():
+    """Eq. 2's double sum equals (sum_j S^L_ij) - (sum_j S^0_ij)."""
+    from oracle.uvprune import similarity_sum, similarity_variation
+    m, n, d, L = 30, 9, 32, 6
+    layers = [_hidden(m, n, d, 10 + l) for l in range(L + 1)]
+    full = similarity_variation(layers, 0, m, m, n)
+    ends = similarity_sum(layers[-1], 0, m, m, n) - similarity_sum(layers[0], 0, m, m, n)
+    np.testing.assert_allclose(full, ends, rtol=0, atol=1e-11)
+
+
+def test_similarity_variation_cancels_positional_component():
+    """Direction only: on the synthetic representations, raw similarity picks pile onto the text-side
+    end of the video; the variation between the first and the 20th layer does not."""
+    from oracle.uvprune import similarity_sum
+    cfg = wl.CONFIGS[0]
+    h0 = wl.hidden_layer(cfg, 0)
+    hL = wl.hidden_layer(cfg, 20)
+    s0 = similarity_sum(h0, 0, cfg.m, cfg.m, cfg.n_text)
+    sL = similarity_sum(hL, 0, cfg.m, cfg.m, cfg.n_text)
+    k = cfg.k_keep
+    raw = select_topk(sL.astype(np.float32), k)
+    var = select_topk((sL - s0).astype(np.float32), k)
+    last_q = 3 * cfg.m // 4
+    assert (raw >= last_q).mean() > 0.6
+    assert (var >= last_q).mean() < 0.45
+    # and the variation finds the tokens whose alignment grew with depth
+    sem = wl.rng_for(cfg.cid, wl.S_HIDDEN, 0).choice(cfg.m, size=max(1, cfg.m // 10), replace=False)
+    assert np.isin(sem, var).mean() > 0.7
