@@ -148,6 +148,37 @@ size_t pvlm_uvprune_workspace_bytes(const pvlm_prune_params *p);
 pvlm_status pvlm_uvprune_select_gather(const pvlm_prune_params *p, void *stream);
 
 /* ------------------------------------------------------------------------
+ * Vision-text similarity signal of UV-Prune on token representations.
+ *
+ * The paper's own pruning criterion (Sec. 4.1): the cosine similarity
+ * S_ij = V_i.X_j / (|V_i||X_j|) between visual token i and text token j in
+ * one early layer of the target (Eq. 1), summed over the text tokens
+ * (the inner sum of Eq. 2):  sim[i] = sum_j S_ij,  i = 0..m-1.
+ * Calling it for the last and for the first layer of the early-layer set and
+ * passing the two results as mass_cur / mass_ref of
+ * pvlm_uvprune_select_gather gives Eq. 2 (which telescopes to the difference
+ * of its two end layers), Eq. 3 and the gather.  A zero vector has similarity
+ * 0 with everything.  fp32 accumulation.
+ *
+ * hidden: bf16 [rows][d] token representations of one layer, row stride
+ * hidden_row_stride elements; visual rows [vis_start, vis_start+m), text
+ * rows [text_start, text_start+n).
+ * Supported: d % 8 == 0, 8 <= d <= 16384; hidden 16-byte aligned, row stride
+ * a multiple of 8; m >= 0, n >= 0.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+  const void *hidden;
+  long long hidden_row_stride;
+  int vis_start, m, text_start, n, d;
+  float *sim;             /* fp32 [m] out */
+  void *workspace;
+  size_t workspace_bytes;
+} pvlm_similarity_params;
+
+size_t pvlm_uvprune_similarity_workspace_bytes(const pvlm_similarity_params *p);
+pvlm_status pvlm_uvprune_similarity(const pvlm_similarity_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
  * Vocab softmax + lossless accept / reject + residual resampling.
  *
  * p_t = softmax(target_logits[t] / temperature), t = 0..gamma;

@@ -4,4 +4,4 @@
 `workloads` draws the seeded synthetic inputs; `build` compiles the library.
 """
 from . import workloads  # noqa: F401
-from .binding import (PvlmError, lib, spec_accept, uvprune_select_gather, verify_attn)  # noqa: F401
+from .binding import (PvlmError, lib, spec_accept, uvprune_select_gather, uvprune_similarity, verify_attn)  # noqa: F401

@@ -66,6 +66,12 @@ class AcceptParams(C.Structure):
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
+class SimilarityParams(C.Structure):
+    _fields_ = [("hidden", C.c_void_p), ("hidden_row_stride", C.c_longlong),
+                ("vis_start", C.c_int), ("m", C.c_int), ("text_start", C.c_int), ("n", C.c_int), ("d", C.c_int),
+                ("sim", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
 class StepParams(C.Structure):
     _fields_ = [("attn", AttnParams), ("prune", PruneParams), ("accept", AcceptParams),
                 ("run_attn", C.c_int), ("run_prune", C.c_int), ("run_accept", C.c_int),
@@ -81,7 +87,7 @@ EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
            "pvlm_verify_attn_workspace_bytes", "pvlm_verify_attn", "pvlm_verify_attn_check",
            "pvlm_uvprune_workspace_bytes", "pvlm_uvprune_select_gather",
            "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept", "pvlm_verify_step",
-           "pvlm_uvprune_select_static")
+           "pvlm_uvprune_select_static", "pvlm_uvprune_similarity_workspace_bytes", "pvlm_uvprune_similarity")
 
 
 def lib() -> C.CDLL:
@@ -105,6 +111,10 @@ def lib() -> C.CDLL:
                 f = getattr(L, name)
                 f.restype = C.c_int
                 f.argtypes = [C.POINTER(st), C.c_void_p]
+            L.pvlm_uvprune_similarity_workspace_bytes.restype = C.c_size_t
+            L.pvlm_uvprune_similarity_workspace_bytes.argtypes = [C.POINTER(SimilarityParams)]
+            L.pvlm_uvprune_similarity.restype = C.c_int
+            L.pvlm_uvprune_similarity.argtypes = [C.POINTER(SimilarityParams), C.c_void_p]
             L.pvlm_uvprune_select_static.restype = C.c_int
             L.pvlm_uvprune_select_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                                      C.c_void_p, C.c_void_p, C.c_void_p]
@@ -347,3 +357,22 @@ def uvprune_select_static(mass_cur, mass_ref, vis_start: int, m: int, k: int, ke
     if st != 0:
         raise PvlmError(st, "pvlm_uvprune_select_static")
     return kept_idx
+
+
+def uvprune_similarity(hidden, vis_start: int, m: int, text_start: int, n: int, *, out=None, workspace=None):
+    """sum_j cos(V_i, X_j) for the m visual rows of one layer's token representations
+    (see pvlm_uvprune_similarity).  hidden: bf16 [rows, d].  Returns fp32 [m]."""
+    _need_cuda(hidden)
+    assert hidden.dtype == torch.bfloat16 and hidden.dim() == 2 and hidden.stride(1) == 1
+    sim = out if out is not None else torch.empty(m, dtype=torch.float32, device=hidden.device)
+    p = SimilarityParams()
+    p.hidden, p.hidden_row_stride = _ptr(hidden), hidden.stride(0)
+    p.vis_start, p.m, p.text_start, p.n, p.d = vis_start, m, text_start, n, hidden.shape[1]
+    p.sim = _ptr(sim)
+    need = lib().pvlm_uvprune_similarity_workspace_bytes(C.byref(p))
+    ws = workspace if workspace is not None else _workspace(hidden.device, "sim", need)
+    p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()
+    st = lib().pvlm_uvprune_similarity(C.byref(p), _stream(hidden.device))
+    if st != 0:
+        raise PvlmError(st, "pvlm_uvprune_similarity")
+    return sim

@@ -128,6 +128,26 @@ pvlm_status pvlm_uvprune_select_gather(const pvlm_prune_params* p, void* stream)
   return launch_uvprune(*p, (cudaStream_t)stream);
 }
 
+static bool similarity_supported(const pvlm_similarity_params* p) {
+  return p->d >= 8 && p->d <= 16384 && p->d % 8 == 0;
+}
+
+size_t pvlm_uvprune_similarity_workspace_bytes(const pvlm_similarity_params* p) {
+  if (!p || p->m < 0 || p->n < 0 || !similarity_supported(p)) return 0;
+  return similarity_workspace(*p);
+}
+
+pvlm_status pvlm_uvprune_similarity(const pvlm_similarity_params* p, void* stream) {
+  if (!p) return PVLM_ERR_INVALID_ARG;
+  if (p->m < 0 || p->n < 0 || p->vis_start < 0 || p->text_start < 0 || p->d < 1) return PVLM_ERR_INVALID_ARG;
+  if (!similarity_supported(p)) return PVLM_ERR_UNSUPPORTED;
+  if (!p->hidden || (p->m > 0 && !p->sim)) return PVLM_ERR_INVALID_ARG;
+  if (!aligned(p->hidden, 16) || p->hidden_row_stride < p->d || p->hidden_row_stride % 8) return PVLM_ERR_INVALID_ARG;
+  const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, similarity_workspace(*p));
+  if (w != PVLM_OK) return w;
+  return launch_similarity(*p, (cudaStream_t)stream);
+}
+
 size_t pvlm_spec_accept_workspace_bytes(const pvlm_accept_params* p) {
   AcceptPlan plan;
   if (!p || !make_accept_plan(*p, plan)) return 0;

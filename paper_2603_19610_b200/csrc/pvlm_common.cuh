@@ -54,6 +54,10 @@ pvlm_status launch_verify_attn(const pvlm_attn_params& p, const AttnPlan& plan, 
 pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s);
 size_t uvprune_workspace(const pvlm_prune_params& p);
 
+// ---- similarity (hidden-state criterion) --------------------------------------------
+size_t similarity_workspace(const pvlm_similarity_params& p);
+pvlm_status launch_similarity(const pvlm_similarity_params& p, cudaStream_t s);
+
 // ---- accept -----------------------------------------------------------------
 struct AcceptPlan {
   int rows;             // 2 * gamma + 1 logit rows per sequence
