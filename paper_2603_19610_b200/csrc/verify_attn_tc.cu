@@ -531,30 +531,35 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               }
             }
           };
-          load_x();
-          PROF_ADD(1)
-          TRACE_T0(5, j)
-          const bool slow = group_or((xmax > kRescaleThreshold) || !ok);
-          PROF_ADD(2)
-          TRACE_T0(6, j)
-          if (slow) {
+          // Attempt 0 converts against the current reference and votes; if the group needs a new reference
+          // the slow path installs it and attempt 1 converts again.  (One copy of the conversion code, and
+          // the slow path's chunk loops stay rolled: it is cold code and should stay small.)
+#pragma unroll 1
+          for (int attempt = 0; attempt < 2; ++attempt) {
+            load_x();
+            if (attempt == 1) break;
+            PROF_ADD(1)
+            TRACE_T0(5, j)
+            const bool slow = group_or((xmax > kRescaleThreshold) || !ok);
+            PROF_ADD(2)
+            TRACE_T0(6, j)
+            if (!slow) break;
             if (group_or(!ok)) { aborted = true; break; }              // uniform across the group
             // ------- slow path: new per-row reference, rescale row sums and the accumulator -------
-#pragma unroll
+#pragma unroll 1
             for (int c = 0; c < NCH; ++c) {
-              {
-                uint32_t raw[16];
-                tmem_ld16(s_addr + c * 16, raw);
-                tmem_wait_ld();
-                reg_fence16(raw);
+              const int cw = (HT && c == NCH - 1) ? 8 : 16;
+              uint32_t raw[16];
+              tmem_ld16(s_addr + c * 16, raw);
+              tmem_wait_ld();
+              reg_fence16(raw);
 #pragma unroll
-                for (int e = 0; e < CW(c); ++e) {
-                  float v = __uint_as_float(raw[e]) * a.scale_log2;
-                  if (need_mask && rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16)) v = -INFINITY;
+              for (int e = 0; e < 16; ++e) {
+                float v = __uint_as_float(raw[e]) * a.scale_log2;
+                if (e >= cw || (need_mask && rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16))) v = -INFINITY;
 #pragma unroll
-                  for (int sh = 16; sh >= 1; sh >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, sh));
-                  if (lane == 0) atomicMax(&newmax_s[c * 16 + e], f2ord(v));
-                }
+                for (int sh = 16; sh >= 1; sh >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, sh));
+                if (lane == 0 && e < cw) atomicMax(&newmax_s[c * 16 + e], f2ord(v));
               }
             }
             group_sync();
@@ -571,7 +576,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               // the accumulator holds this group's earlier tiles: wait until the last of them has been added
               ok &= mbar_wait(bar(P_FREE + g), ((j >> 1) - 1) & 1, s_abort);
               tc_fence_after();
-#pragma unroll
+#pragma unroll 1
               for (int c = 0; c < NCH; ++c) {
                 uint32_t o[16];
                 tmem_ld16(tmem_O + lane_addr + g * NRP + c * 16, o);
@@ -583,8 +588,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               }
               tmem_wait_st();
             }
-            load_x();                                  // scores against the new reference
           }
+          if (aborted) break;
           PROF_ADD(3)
           // the score buffer is no longer needed: let the issuer refill it
           tc_fence_before();

@@ -200,3 +200,17 @@ def test_timeout_status_is_reported_from_the_workspace_word():
     assert binding.lib().pvlm_verify_attn_check(C.byref(p), st) == 6
     assert binding.lib().pvlm_verify_attn(C.byref(p), st) == 0                                    # a new call clears it
     assert binding.lib().pvlm_verify_attn_check(C.byref(p), st) == 0
+
+
+def test_tensor_core_path_is_deterministic():
+    """Same inputs twice through the tcgen05 kernels: bitwise equal O, lse and mass (no float atomics,
+    fixed-order merges)."""
+    qb, kb, vb = wl.make_qkv(40, 8, 128, 13, 6013, sink=True, seed=123)
+    q, k, v = bf16_cuda(qb), bf16_cuda(kb), bf16_cuda(vb)
+    a = binding.verify_attn(q, k, v, 6000, want_mass=True)
+    a = [x.clone() for x in a]
+    for _ in range(3):
+        b = binding.verify_attn(q, k, v, 6000, want_mass=True)
+        torch.cuda.synchronize()
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
