@@ -196,7 +196,11 @@ pvlm_status pvlm_uvprune_similarity(const pvlm_similarity_params *p, void *strea
  * packed [batch][...].  Full-probability outputs, if requested, use the same
  * strides as the logits (so they need non-zero batch strides).
  *
- * Supported: 1 <= gamma <= 64; 1 <= V < 2^31; 1 <= batch <= 65535.  Rows are
+ * gamma = 0 is plain sampling: nothing is verified, one token is drawn from
+ * p_0 with uniform u_0 (the draft model's own decoding step uses the call
+ * this way on its logits); draft_logits and draft_tokens may then be NULL.
+ *
+ * Supported: 0 <= gamma <= 64; 1 <= V < 2^31; 1 <= batch <= 65535.  Rows are
  * read with 16-byte loads when the logit base pointers are 16-byte aligned
  * and all logit strides are multiples of 4 elements, else element by element.
  * ---------------------------------------------------------------------- */
@@ -265,6 +269,21 @@ typedef struct {
 } pvlm_step_params;
 
 pvlm_status pvlm_verify_step(const pvlm_step_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Draft window size from measured forward times (host arithmetic, no GPU).
+ *
+ * The window equals the pruned speed ratio c* = T_p / T_q(alpha) (paper
+ * Eq. 6).  c* is rarely an integer; the paper calls rounding down the wiser
+ * choice when the window is aggressive relative to the mean accepted length
+ * and rounding up the sensible one for narrow windows with high accepted
+ * lengths (Appendix A, "Window Size Selection"), and leaves the choice to the
+ * user; the five window sizes it uses itself all equal c* rounded to the
+ * nearest integer.  mode: 0 = nearest, 1 = down, 2 = up.  Never below 1.
+ * Returns 0 if a time is not positive or the mode is unknown.
+ * ---------------------------------------------------------------------- */
+enum { PVLM_ROUND_NEAREST = 0, PVLM_ROUND_DOWN = 1, PVLM_ROUND_UP = 2 };
+int pvlm_window_size(double t_target, double t_draft, int mode);
 
 /* ------------------------------------------------------------------------
  * Top-K selection that needs no caller-side scratch allocation.

@@ -15,4 +15,4 @@ tests); none is "parity unpinned".
 from .attention import bf16_bits_to_f64, verify_attn  # noqa: F401
 from .uvprune import (variation_score, select_topk, gather_rows, cosine_similarity, similarity_sum,  # noqa: F401
                       similarity_variation)
-from .accept import softmax64, spec_accept, window_size  # noqa: F401
+from .accept import softmax64, spec_accept, window_size, window_size_rounded  # noqa: F401

@@ -88,6 +88,16 @@ def window_size(T_p: float, T_q: float) -> float:
     return T_p / T_q
 
 
+def window_size_rounded(T_p: float, T_q: float, mode: str = "nearest") -> int:
+    """Integer window from c* = T_p / T_q.  The paper leaves the rounding direction to the user (down for
+    windows that are aggressive relative to the accepted length, up for narrow windows with high accepted
+    lengths, Appendix A); the five windows it uses itself equal c* rounded to the nearest integer."""
+    import math
+    c = window_size(T_p, T_q)
+    g = {"nearest": math.floor(c + 0.5), "down": math.floor(c + 1e-9), "up": math.ceil(c - 1e-9)}[mode]
+    return max(1, int(g))
+
+
 def spec_accept_trials(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0):
     """The same rule as `spec_accept`, applied to B independent trials that
     share one set of logits: draft_tokens int [B, gamma], uniforms fp32

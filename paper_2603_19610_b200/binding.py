@@ -87,7 +87,7 @@ EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
            "pvlm_verify_attn_workspace_bytes", "pvlm_verify_attn", "pvlm_verify_attn_check",
            "pvlm_uvprune_workspace_bytes", "pvlm_uvprune_select_gather",
            "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept", "pvlm_verify_step",
-           "pvlm_uvprune_select_static", "pvlm_uvprune_similarity_workspace_bytes", "pvlm_uvprune_similarity")
+           "pvlm_uvprune_select_static", "pvlm_uvprune_similarity_workspace_bytes", "pvlm_uvprune_similarity", "pvlm_window_size")
 
 
 def lib() -> C.CDLL:
@@ -376,3 +376,37 @@ def uvprune_similarity(hidden, vis_start: int, m: int, text_start: int, n: int, 
     if st != 0:
         raise PvlmError(st, "pvlm_uvprune_similarity")
     return sim
+
+
+def sample(logits, uniforms, temperature: float = 1.0, *, workspace=None):
+    """Draw one token per row from softmax(logits / temperature) by inverse CDF: pvlm_spec_accept with
+    gamma = 0 (nothing to verify), the form the draft model's own decoding step uses.
+    logits fp32 [B, V] (or [V]), uniforms fp32 [B] (or scalar tensor).  Returns int32 tokens [B]."""
+    _need_cuda(logits, uniforms)
+    lg = logits if logits.dim() == 2 else logits[None]
+    B, V = lg.shape
+    assert lg.dtype == torch.float32 and lg.stride(1) == 1 and uniforms.dtype == torch.float32
+    dev = lg.device
+    n_accept = torch.empty(B, dtype=torch.int32, device=dev)
+    out = torch.empty((B, 1), dtype=torch.int32, device=dev)
+    p = AcceptParams()
+    p.target_logits = _ptr(lg)
+    p.target_row_stride, p.target_batch_stride = V, lg.stride(0)
+    p.uniforms = _ptr(uniforms.contiguous())
+    p.batch, p.gamma, p.V, p.temperature = B, 0, V, float(temperature)
+    p.n_accept, p.out_tokens = _ptr(n_accept), _ptr(out)
+    need = lib().pvlm_spec_accept_workspace_bytes(C.byref(p))
+    ws = workspace if workspace is not None else _workspace(dev, "accept", need)
+    p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()
+    st = lib().pvlm_spec_accept(C.byref(p), _stream(dev))
+    if st != 0:
+        raise PvlmError(st, "pvlm_spec_accept")
+    return out[:, 0]
+
+
+def window_size(t_target: float, t_draft: float, mode: str = "nearest") -> int:
+    """Draft window from measured forward times (see pvlm_window_size); mode nearest / down / up."""
+    f = lib().pvlm_window_size
+    f.restype = C.c_int
+    f.argtypes = [C.c_double, C.c_double, C.c_int]
+    return int(f(float(t_target), float(t_draft), {"nearest": 0, "down": 1, "up": 2}[mode]))

@@ -1,6 +1,8 @@
 // C-ABI entry points: host-side argument validation, workspace queries, dispatch.
 #include "pvlm_common.cuh"
 
+#include <cmath>
+
 namespace pvlm {
 
 static thread_local int g_last_cuda_error = 0;
@@ -156,14 +158,14 @@ size_t pvlm_spec_accept_workspace_bytes(const pvlm_accept_params* p) {
 
 pvlm_status pvlm_spec_accept(const pvlm_accept_params* p, void* stream) {
   if (!p) return PVLM_ERR_INVALID_ARG;
-  if (p->gamma < 1 || p->V < 1 || p->batch < 1) return PVLM_ERR_INVALID_ARG;
-  if (!p->target_logits || !p->draft_logits || !p->draft_tokens || !p->uniforms || !p->n_accept || !p->out_tokens)
-    return PVLM_ERR_INVALID_ARG;
+  if (p->gamma < 0 || p->V < 1 || p->batch < 1) return PVLM_ERR_INVALID_ARG;
+  if (!p->target_logits || !p->uniforms || !p->n_accept || !p->out_tokens) return PVLM_ERR_INVALID_ARG;
+  if (p->gamma > 0 && (!p->draft_logits || !p->draft_tokens)) return PVLM_ERR_INVALID_ARG;
   AcceptPlan plan;
   if (!make_accept_plan(*p, plan)) return PVLM_ERR_UNSUPPORTED;
   if (p->batch > 65535) return PVLM_ERR_UNSUPPORTED;
   if (!aligned(p->target_logits, 4) || !aligned(p->draft_logits, 4)) return PVLM_ERR_INVALID_ARG;
-  if (p->target_row_stride < p->V || p->draft_row_stride < p->V) return PVLM_ERR_INVALID_ARG;
+  if (p->target_row_stride < p->V || (p->gamma > 0 && p->draft_row_stride < p->V)) return PVLM_ERR_INVALID_ARG;
   if (p->batch > 1) {
     // batch stride 0 = every sequence reads the same logits
     if (p->target_batch_stride != 0 && (p->target_batch_stride < (long long)(p->gamma + 1) * p->target_row_stride)) return PVLM_ERR_INVALID_ARG;
@@ -211,7 +213,7 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     }
   }
   if (p->run_accept) {
-    if (c.gamma < 1 || c.V < 1 || c.batch < 1) return PVLM_ERR_INVALID_ARG;
+    if (c.gamma < 0 || c.V < 1 || c.batch < 1) return PVLM_ERR_INVALID_ARG;
     if (p->h_target_logits || p->h_draft_logits) {
       if (c.target_row_stride != c.V || c.draft_row_stride != c.V) return PVLM_ERR_UNSUPPORTED;
       if (c.batch > 1 && (c.target_batch_stride != (long long)(c.gamma + 1) * c.V ||
@@ -257,6 +259,19 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
   if (overlap && p->run_attn && p->h_o && ok()) e = cudaStreamWaitEvent(s, eb, 0);   // `stream` now also covers the o download
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   return PVLM_OK;
+}
+
+int pvlm_window_size(double t_target, double t_draft, int mode) {
+  if (!(t_target > 0.0) || !(t_draft > 0.0)) return 0;
+  const double c = t_target / t_draft;
+  double g;
+  if (mode == PVLM_ROUND_NEAREST) g = floor(c + 0.5);
+  else if (mode == PVLM_ROUND_DOWN) g = floor(c + 1e-9);
+  else if (mode == PVLM_ROUND_UP) g = ceil(c - 1e-9);
+  else return 0;
+  if (g < 1.0) g = 1.0;
+  if (g > 1e9) g = 1e9;
+  return (int)g;
 }
 
 }  // extern "C"

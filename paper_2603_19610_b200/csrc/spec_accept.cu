@@ -321,7 +321,7 @@ __global__ void __launch_bounds__(256) write_probs_kernel(const AccArgs a) {
 }  // namespace
 
 bool make_accept_plan(const pvlm_accept_params& p, AcceptPlan& plan) {
-  if (p.gamma < 1 || p.gamma > 64 || p.V < 1 || p.batch < 1) return false;
+  if (p.gamma < 0 || p.gamma > 64 || p.V < 1 || p.batch < 1) return false;
   plan.rows = 2 * p.gamma + 1;
   plan.stat_chunk = kStatChunk;
   plan.n_stat_chunks = ceil_div(p.V, kStatChunk);

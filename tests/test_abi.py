@@ -95,3 +95,11 @@ def test_no_cpu_fallback():
     q = torch.zeros(2, 4, 64, dtype=torch.bfloat16)
     with pytest.raises(RuntimeError):
         binding.verify_attn(q, torch.zeros(10, 1, 64, dtype=torch.bfloat16), torch.zeros(10, 1, 64, dtype=torch.bfloat16), 8)
+
+
+def test_window_size_host_function_matches_oracle():
+    from oracle.accept import window_size_rounded
+    for tp, tq in [(420, 46.6), (203, 39.8), (78.3, 25.8), (78.3, 46.6), (420, 78), (10, 50), (63.7, 39.8)]:
+        for mode in ("nearest", "down", "up"):
+            assert binding.window_size(tp, tq, mode) == window_size_rounded(tp, tq, mode)
+    assert binding.window_size(0, 1) == 0 and binding.window_size(1, -1) == 0

@@ -149,3 +149,38 @@ def test_chi_square_on_gpu_path():
         if n_gpu[b] != n_ref[b]:
             t = min(n_gpu[b], n_ref[b])
             assert abs(float(u[b, t]) - p[t, x[b, t]] / q[t, x[b, t]]) <= 1e-5
+
+
+def test_sample_gamma_zero_matches_inverse_cdf():
+    """gamma = 0 through the same entry point is plain sampling (the draft's own decoding step): the token is
+    the oracle's inverse-CDF draw from softmax(logits / T); tokens that differ must sit on a CDF boundary."""
+    from oracle.accept import inverse_cdf
+    rng = np.random.default_rng(31)
+    for V, B, T in [(151_936, 6, 1.0), (4099, 9, 0.7), (16, 64, 1.3), (1, 3, 1.0)]:
+        lg = (2.0 * rng.standard_normal((B, V))).astype(np.float32)
+        u = wl.unit_uniforms(rng, B)
+        tok = binding.sample(torch.from_numpy(lg).cuda(), torch.from_numpy(u).cuda(), T).cpu().numpy()
+        for b in range(B):
+            p = softmax64(lg[b][None], T)[0]
+            ref = inverse_cdf(p, float(u[b]))
+            if tok[b] != ref:
+                c = np.cumsum(p)
+                lo, hi = sorted((int(tok[b]), int(ref)))
+                assert hi - lo == 1 and abs(c[lo] - float(u[b]) * c[-1]) <= 1e-6, (V, b, tok[b], ref)
+    o = oracle_accept(lg[0][None], np.zeros((0, V), np.float32), np.zeros(0, np.int32), u[:1])
+    assert o["n_accept"] == 0 and o["out_tokens"][0] == binding.sample(torch.from_numpy(lg[0]).cuda(), torch.from_numpy(u[:1]).cuda()).item()
+
+
+def test_sample_gamma_zero_chi_square():
+    """4e5 draws from one row (stride-0 batch): counts follow softmax (df = 15, p-value 1e-4)."""
+    V, B = 16, 400_000
+    rng = np.random.default_rng(77)
+    lg = (1.5 * rng.standard_normal(V)).astype(np.float32)
+    u = wl.unit_uniforms(np.random.Generator(np.random.Philox(key=99)), B)
+    lg_d, step = torch.from_numpy(lg).cuda(), 50_000                      # one call takes at most 65535 rows
+    tok = np.concatenate([binding.sample(lg_d[None].expand(step, -1), torch.from_numpy(u[s:s + step]).cuda()).cpu().numpy()
+                          for s in range(0, B, step)])
+    counts = np.bincount(tok, minlength=V).astype(np.float64)
+    p = softmax64(lg[None])[0]
+    stat = ((counts - B * p) ** 2 / (B * p)).sum()
+    assert stat < chi2.isf(1e-4, V - 1), stat

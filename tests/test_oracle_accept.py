@@ -222,3 +222,25 @@ def test_window_rule_printed_examples():
         c = window_size(tp, tq)
         tol = 0.5 if printed == round(printed) and "." not in line.split()[2] else 0.1
         assert abs(c - printed) <= tol, (tp, tq, c, printed)
+
+
+def test_window_choice_reproduces_the_papers_gammas():
+    """Nearest-integer rounding of c* on the paper's printed forward times gives the window sizes the
+    paper uses for its five model pairs; the other two modes bracket it."""
+    from oracle.accept import window_size_rounded
+    for line in open(os.path.join(GOLD, "window_choice.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        tp, tq, gamma = line.split()
+        assert window_size_rounded(float(tp), float(tq)) == int(gamma), line
+        assert window_size_rounded(float(tp), float(tq), "down") <= int(gamma) <= window_size_rounded(float(tp), float(tq), "up")
+    assert window_size_rounded(420, 78, "down") == 5 and window_size_rounded(420, 47, "down") == 8
+    assert window_size_rounded(420, 47, "up") == 9 and window_size_rounded(10, 50) == 1
+
+
+def test_gamma_zero_is_plain_sampling():
+    rng = np.random.default_rng(0)
+    tl = rng.standard_normal((1, 50)).astype(np.float32)
+    r = spec_accept(tl, np.zeros((0, 50), np.float32), np.zeros(0, np.int32), np.array([0.37], np.float32))
+    assert r["n_accept"] == 0 and r["out_tokens"].shape == (1,)
+    assert r["out_tokens"][0] == inverse_cdf(softmax64(tl)[0], 0.37)
