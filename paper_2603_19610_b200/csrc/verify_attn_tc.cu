@@ -37,13 +37,13 @@ namespace pvlm {
 namespace {
 
 constexpr int kTile = 128;                 // keys per tile
-constexpr int kKStages = 2, kVStages = 2;
 constexpr int kBoxBytes = kTile * 128;     // one 64-channel box of a 128-key tile: 16 KB
 constexpr int kTileBytes = 2 * kBoxBytes;  // 32 KB
 constexpr int kSoftmaxThreads = 256;
 constexpr int kGroupThreads = 128;         // one softmax group
 constexpr int kThreads = 128 + kSoftmaxThreads;   // warpgroup 0: TMA + MMA (+2 idle warps); warpgroups 1, 2: softmax
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSuspendHintNs = 20000;        // upper bound of one sleep inside try_wait
+constexpr uint64_t kWaitLimitNs = 1000000000ull;   // a wait that lasts a second has failed
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 constexpr float kNegBig = -1.0e30f;        // "no key seen yet" reference: finite, so differences never give NaN
 
@@ -76,9 +76,15 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait: false if the phase did not complete within the spin limit or another thread gave up.
-// A first non-blocking test_wait serves the common case of a phase that completed long ago (the
-// potentially-suspending try_wait costs a couple of hundred cycles even then).
+// Bounded wait: false if the phase did not complete within the time limit or another thread gave up.
+// A first non-blocking test_wait serves the common case of a phase that completed long ago.  After
+// that the thread sleeps inside try_wait (suspend-time hint) instead of polling: 300 spinning threads
+// per SM cost enough power to pull the SM clock down under the board's power cap.
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   uint32_t ok;
   asm volatile(
@@ -89,16 +95,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       : "r"(bar), "r"(parity)
       : "memory");
   if (ok) return true;
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+  const uint64_t t0 = global_ns();
+  for (;;) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     if (ok) return true;
     if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) break;
   }
   *abort_flag = 1;
   return false;
@@ -148,6 +156,16 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
+}
+// One lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -203,6 +221,9 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
 // ---------------------------------------------------------------------------------------------
 // The kernel.  NRP = query rows per KV head padded to a multiple of 16 (MMA N), NRP <= 96.
 // ---------------------------------------------------------------------------------------------
+// K and V tiles share one ring of 32 KB slots, filled and drained in the order the issuer consumes them.
+// Five slots fit beside Q and the two P buffers up to 80 padded rows.
+__host__ __device__ constexpr int ring_slots(int nrp) { return nrp <= 80 ? 5 : 4; }
 __host__ __device__ constexpr int s_bufs(int nrp) { return (512 - 2 * nrp) / nrp >= 4 ? 4 : (512 - 2 * nrp) / nrp; }
 
 // HT: the last 16-column chunk holds at most 8 real query rows, so only its first 8 columns are processed.
@@ -214,6 +235,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   constexpr int QBOX = NRP * 128;          // bytes of one 64-channel box of Q
   constexpr int PBYTES = NRP * 256;        // one P buffer: NRP/8 row groups x 2048 B
   constexpr int NSB = s_bufs(NRP);         // score buffers in TMEM
+  constexpr int NS = ring_slots(NRP);      // K/V ring slots
   constexpr uint32_t NEED = (2 + NSB) * NRP;
   constexpr uint32_t TMEM_COLS = NEED <= 32 ? 32 : NEED <= 64 ? 64 : NEED <= 128 ? 128 : NEED <= 256 ? 256 : 512;
   constexpr uint32_t IDESC_QK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NRP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
@@ -222,20 +244,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  unsigned char* sK = smem;
-  unsigned char* sV = sK + kKStages * kTileBytes;
-  unsigned char* sQ = sV + kVStages * kTileBytes;
+  unsigned char* sRing = smem;
+  unsigned char* sQ = sRing + NS * kTileBytes;
   unsigned char* sP = sQ + 2 * QBOX;                                  // one P buffer per softmax group
   float* s_m = reinterpret_cast<float*>(sP + 2 * PBYTES);            // [2][128] running reference per group
   float* s_fac = s_m + 256;                                           // [2][128] rescale factors (slow path)
   int* s_newmax = reinterpret_cast<int*>(s_fac + 256);               // [2][128]
-  float* s_lsum = reinterpret_cast<float*>(s_newmax + 256);          // [2][4][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(s_lsum + 1024);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_newmax + 256);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 32);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
-  enum { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, P_FULL = 8, P_FREE = 10, Q_READY = 12, O_FULL = 13, O_FREE = 14,
-         S_FULL = 16, S_FREE = 20 };
+  // K_FULL and P_FULL are indexed by tile % 4.  P_FULL(j) completes when the group's 128 threads have stored
+  // P(j) AND the V tile has landed (the producer arrives on it with the tile's byte count), so the issuer
+  // needs one wait per MMA group.  EMPTY(slot) is committed behind the MMAs that read the slot.
+  // There is no "score buffer free" barrier: score tile j+lookahead is issued after P_FULL(j-1) was seen,
+  // and a group arrives there only after it has read its scores, which frees every buffer up to j-1.
+  enum { K_FULL = 0, P_FULL = 4, P_FREE = 8, Q_READY = 10, O_FULL = 11, O_FREE = 12, S_FULL = 13, EMPTY = 17 };
   auto bar = [&](int i) { return smem_addr(bars + i); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -247,12 +271,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int item_first = (int)(f_begin / Tt);
 
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1);
-      mbar_init(bar(V_FULL + i), 1); mbar_init(bar(V_EMPTY + i), 1);
-      mbar_init(bar(P_FULL + i), kGroupThreads); mbar_init(bar(P_FREE + i), 1);
-    }
-    for (int i = 0; i < NSB; ++i) { mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), kGroupThreads); }
+    for (int i = 0; i < 4; ++i) { mbar_init(bar(K_FULL + i), 1); mbar_init(bar(P_FULL + i), kGroupThreads + 1); }
+    for (int i = 0; i < 2; ++i) mbar_init(bar(P_FREE + i), 1);
+    for (int i = 0; i < NSB; ++i) mbar_init(bar(S_FULL + i), 1);
+    for (int i = 0; i < NS; ++i) mbar_init(bar(EMPTY + i), 1);
     mbar_init(bar(Q_READY), kSoftmaxThreads);
     mbar_init(bar(O_FULL), 1);
     mbar_init(bar(O_FREE), kSoftmaxThreads);
@@ -278,63 +300,58 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (warp < 4) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == 0) {
       // =========================== TMA producer ===========================
+      // Walks the same loop as the MMA issuer, so tiles enter the ring in the order they leave it:
+      // per segment K(0..lookahead), V(0), K(lookahead+1), V(1), ...  It runs ahead across segment
+      // boundaries as far as free slots allow.
       if (lane == 0) {
         PROF_DECL
-        uint32_t jk = 0, jv = 0;                 // K and V rings advance separately: K leads by the score look-ahead
-        const uint32_t total = (uint32_t)(f_end - f_begin);
-        auto coords = [&](uint32_t j, int& kvh, int& tile, int& layer) {
-          const long long f = f_begin + j;
-          const int item = (int)(f / Tt);
-          tile = (int)(f - (long long)item * Tt);
-          layer = item / a.Hkv;
-          kvh = item - layer * a.Hkv;
-        };
-        // The MMA issuer runs the score MMAs `lookahead` tiles ahead of the PV MMAs, so V(j) may only be
-        // waited for once K has been issued through tile j+lookahead (otherwise the issuer would wait
-        // for a K tile that this thread, blocked on a V slot, never sends).
-        while (jk < total || jv < total) {
+        uint32_t u = 0;                          // loads issued so far (ring position)
+        uint32_t jt = 0;
+        bool ok = true;
+        auto load = [&](const CUtensorMap* map, uint32_t full_bar, long long f) -> bool {
+          const uint32_t slot = u % NS;
           PROF_START
-          // K tiles that must be on their way before PV(jv) can be issued; never past the end of
-          // jv's segment, because the next segment's score MMAs wait for this segment's epilogue
-          uint32_t need_k = total;
-          if (jv < total) {
-            const long long fv = f_begin + jv;
-            const long long seg_end_j = min(f_end, (fv / Tt + 1) * (long long)Tt) - f_begin;
-            need_k = (uint32_t)min((long long)jv + a.lookahead + 1, seg_end_j);
-          }
-          if (jk < total && jk < need_k) {
-            const uint32_t ks = jk % kKStages;
-            int kvh, tile, layer;
-            coords(jk, kvh, tile, layer);
-            // slot ks was read by the score MMAs of tile jk-2: their completion is the S_FULL phase of that tile
-            if (jk >= kKStages && !mbar_wait(bar(S_FULL + (jk - kKStages) % NSB), ((jk - kKStages) / NSB) & 1, s_abort)) break;
-            PROF_ADD(0)
-            mbar_expect_tx(bar(K_FULL + ks), kTileBytes);
-            tma_load_4d(smem_addr(sK + ks * kTileBytes), &tm_k, bar(K_FULL + ks), 0, kvh, tile * kTile, layer);
-            tma_load_4d(smem_addr(sK + ks * kTileBytes + kBoxBytes), &tm_k, bar(K_FULL + ks), 64, kvh, tile * kTile, layer);
-            ++jk;
-            continue;
-          }
-          const uint32_t vs = jv % kVStages;
-          int kvh, tile, layer;
-          coords(jv, kvh, tile, layer);
-          // slot vs was read by the PV MMAs of tile jv-2: their completion is that group's P_FREE phase
-          if (jv >= kVStages && !mbar_wait(bar(P_FREE + ((jv - kVStages) & 1)), ((jv - kVStages) >> 1) & 1, s_abort)) break;
-          PROF_ADD(1)
-          mbar_expect_tx(bar(V_FULL + vs), kTileBytes);
-          tma_load_4d(smem_addr(sV + vs * kTileBytes), &tm_v, bar(V_FULL + vs), 0, kvh, tile * kTile, layer);
-          tma_load_4d(smem_addr(sV + vs * kTileBytes + kBoxBytes), &tm_v, bar(V_FULL + vs), 64, kvh, tile * kTile, layer);
-          ++jv;
+          if (u >= NS && !mbar_wait(bar(EMPTY + slot), ((u / NS) - 1) & 1, s_abort)) return false;
+          PROF_ADD(0)
+          const int item = (int)(f / Tt), tile = (int)(f - (long long)item * Tt);
+          const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
+          const uint32_t dst = smem_addr(sRing + slot * kTileBytes);
+          mbar_expect_tx(full_bar, kTileBytes);
+          tma_load_4d(dst, map, full_bar, 0, kvh, tile * kTile, layer);
+          tma_load_4d(dst + kBoxBytes, map, full_bar, 64, kvh, tile * kTile, layer);
+          ++u;
           PROF_ADD(2)
+          return true;
+        };
+        for (long long f = f_begin; f < f_end && ok;) {
+          const int item = (int)(f / Tt);
+          const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
+          const int n = (int)(seg_end - f);
+          int issued = 0;
+          for (int i = 0; i < n && ok; ++i) {
+            while (ok && issued < n && issued <= i + a.lookahead) {
+              ok = load(&tm_k, bar(K_FULL + ((jt + issued) & 3)), f + issued);
+              ++issued;
+            }
+            if (ok) ok = load(&tm_v, bar(P_FULL + ((jt + i) & 3)), f + i);
+          }
+          jt += n;
+          f = seg_end;
         }
         if (blockIdx.x == 0) PROF_DUMP(4)
       }
     } else if (warp == 1) {
       // =========================== MMA issuer ===========================
-      // One thread issues both MMA streams in order: score tiles run `lookahead` tiles ahead of the
-      // PV tiles, and the fixed interleave keeps the two softmax groups half a period apart.
-      if (lane == 0) {
+      // The whole warp walks the loop (so tile counters, barrier addresses and descriptors are
+      // warp-uniform values) and one elected lane issues the MMAs and commits.  Score tiles run
+      // `lookahead` tiles ahead of the PV tiles; the fixed interleave of the two streams keeps the
+      // two softmax groups half a period apart.
+      {
         const uint32_t q_base = smem_addr(sQ);
+        // descriptor constants: only the 14-bit start-address field changes from MMA to MMA
+        const uint64_t desc_k0 = make_desc(smem_addr(sRing), 16, 1024, 2), desc_q0 = make_desc(q_base, 16, 1024, 2);
+        const uint64_t desc_v0 = make_desc(smem_addr(sRing), kBoxBytes, 1024, 2), desc_p0 = make_desc(smem_addr(sP), 128, 2048, 0);
+        uint32_t u = 0;            // ring position (same sequence as the producer's)
         bool ok = true;
         PROF_DECL
         uint32_t jt = 0;           // tiles issued by this CTA so far (ring phases run across segments)
@@ -351,22 +368,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           a.status[141] = (int)((c2 - c1) / 64);
         }
 #endif
+        auto wait_all = [&](uint32_t b, uint32_t parity) -> bool {     // a vote makes the outcome provably warp-uniform
+          return __all_sync(0xffffffffu, mbar_wait(b, parity, s_abort));
+        };
         auto issue_qk = [&](uint32_t j) -> bool {
-          const uint32_t ks = j % kKStages, sb = j % NSB;
+          const uint32_t slot = u % NS, sb = j % NSB;
+          ++u;
           PROF_START
-          if (!mbar_wait(bar(K_FULL + ks), (j / kKStages) & 1, s_abort)) return false;
+          if (!wait_all(bar(K_FULL + (j & 3)), (j >> 2) & 1)) return false;
           PROF_ADD(0)
-          if (j >= NSB && !mbar_wait(bar(S_FREE + sb), ((j / NSB) - 1) & 1, s_abort)) return false;
-          PROF_ADD(1)
           TRACE(0, j)
           tc_fence_after();
-          const uint32_t k_base = smem_addr(sK + ks * kTileBytes);
+          const uint64_t dk = desc_k0 + (uint64_t)((slot * kTileBytes) >> 4);
+          const uint32_t d_tmem = tmem_S + sb * NRP;
+          if (elect_one()) {
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32, qoff = (kk >> 2) * QBOX + (kk & 3) * 32;
-            tc_mma(tmem_S + sb * NRP, make_desc(k_base + off, 16, 1024, 2), make_desc(q_base + qoff, 16, 1024, 2), IDESC_QK, kk > 0);
+            for (int kk = 0; kk < 8; ++kk) {
+              const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32, qoff = (kk >> 2) * QBOX + (kk & 3) * 32;
+              tc_mma(d_tmem, dk + (off >> 4), desc_q0 + (qoff >> 4), IDESC_QK, kk > 0);
+            }
+            tc_commit(bar(S_FULL + sb));
+            tc_commit(bar(EMPTY + slot));
           }
-          tc_commit(bar(S_FULL + sb));          // also frees the K slot (the K producer waits on this phase)
+          __syncwarp();
           PROF_ADD(2)
           TRACE(1, j)
           return true;
@@ -375,7 +399,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const int item = (int)(f / Tt);
           const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
           const int n = (int)(seg_end - f);
-          if (!mbar_wait(bar(Q_READY), seg & 1, s_abort)) { ok = false; break; }
+          if (!wait_all(bar(Q_READY), seg & 1)) { ok = false; break; }
           tc_fence_after();
           int issued = 0;                                  // score tiles of this segment already issued
           for (int i = 0; i < n; ++i) {
@@ -385,31 +409,36 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               ++issued;
             }
             if (!ok) break;
-            const uint32_t vs = j % kVStages, g = j & 1;
+            const uint32_t slot = u % NS, g = j & 1;
+            ++u;
             PROF_START
-            if (i == 0 && seg > 0 && !mbar_wait(bar(O_FREE), (seg - 1) & 1, s_abort)) { ok = false; break; }
+            if (i == 0 && seg > 0 && !wait_all(bar(O_FREE), (seg - 1) & 1)) { ok = false; break; }
             PROF_ADD(3)
-            if (!mbar_wait(bar(V_FULL + vs), (j / kVStages) & 1, s_abort)) { ok = false; break; }
-            PROF_ADD(4)
-            if (!mbar_wait(bar(P_FULL + g), (j >> 1) & 1, s_abort)) { ok = false; break; }
+            if (!wait_all(bar(P_FULL + (j & 3)), (j >> 2) & 1)) { ok = false; break; }     // P stored and V landed
             PROF_ADD(5)
             TRACE(2, j)
             tc_fence_after();
-            const uint32_t v_base = smem_addr(sV + vs * kTileBytes), p_base = smem_addr(sP + g * PBYTES);
+            const uint64_t dv = desc_v0 + (uint64_t)((slot * kTileBytes) >> 4), dp = desc_p0 + (uint64_t)((g * PBYTES) >> 4);
+            const uint32_t d_tmem = tmem_O + g * NRP;
+            const uint32_t acc0 = i >= 2;                  // each group's accumulator starts afresh in every segment
+            if (elect_one()) {
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-              tc_mma(tmem_O + g * NRP, make_desc(v_base + kk * 2048, kBoxBytes, 1024, 2), make_desc(p_base + kk * 256, 128, 2048, 0),
-                     IDESC_PV, (i >= 2 || kk > 0));      // each group's accumulator starts afresh in every segment
-            tc_commit(bar(P_FREE + g));          // also frees the V slot (the V producer waits on this phase)
+              for (int kk = 0; kk < 8; ++kk)
+                tc_mma(d_tmem, dv + (uint64_t)((kk * 2048) >> 4), dp + (uint64_t)((kk * 256) >> 4), IDESC_PV, (kk > 0) ? 1u : acc0);
+              tc_commit(bar(P_FREE + g));
+              tc_commit(bar(EMPTY + slot));
+            }
+            __syncwarp();
             PROF_ADD(6)
             TRACE(3, j)
           }
           if (!ok) break;
-          tc_commit(bar(O_FULL));
+          if (elect_one()) tc_commit(bar(O_FULL));
+          __syncwarp();
           jt += n;
           f = seg_end;
         }
-        if (blockIdx.x == 0) PROF_DUMP(16)
+        if (blockIdx.x == 0 && lane == 0) PROF_DUMP(16)
       }
     } else if (warp >= 4) {
       // =========================== softmax warps ===========================
@@ -425,6 +454,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       float* m_s = s_m + g * 128;
       float* fac_s = s_fac + g * 128;
       int* newmax_s = s_newmax + g * 128;
+      // per-warp row sums of the epilogue live in the first row group (2 KB) of the group's P buffer: the last
+      // PV of the segment has been waited for by then, and every tile rewrites that row group
+      float* lsum_s = reinterpret_cast<float*>(sP + g * PBYTES);
       float l_loc[NRP];
       uint32_t jt = 0;
       int seg = 0;
@@ -591,9 +623,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           }
           if (aborted) break;
           PROF_ADD(3)
-          // the score buffer is no longer needed: let the issuer refill it
-          tc_fence_before();
-          mbar_arrive(bar(S_FREE + sb));
           // ---- probabilities, running sums, bf16 P in the MN-major core-matrix layout ----
           if (i >= 2) ok &= mbar_wait(bar(P_FREE + g), ((j >> 1) - 1) & 1, s_abort);
           PROF_ADD(4)
@@ -617,7 +646,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           }
           PROF_ADD(5)
           fence_proxy_async();
-          mbar_arrive(bar(P_FULL + g));
+          tc_fence_before();                    // the score buffer has been read: this arrival also releases it
+          mbar_arrive(bar(P_FULL + (j & 3)));
           PROF_ADD(6)
           TRACE_T0(8, j)
         }
@@ -647,11 +677,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           float v = l_loc[k];
 #pragma unroll
           for (int sh = 16; sh >= 1; sh >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sh);
-          if (lane == 0) s_lsum[(g * 4 + q4) * 128 + k] = v;
+          if (lane == 0) lsum_s[q4 * 128 + k] = v;
         }
         group_sync();
         if (t < NRP) {
-          const float* ls = s_lsum + g * 512;
+          const float* ls = lsum_s;
           const float l = ((ls[t] + ls[128 + t]) + ls[256 + t]) + ls[384 + t];
           a.part_ml[(slot * NRP + t) * 2] = has_tiles ? m_s[t] : kNegBig;
           a.part_ml[(slot * NRP + t) * 2 + 1] = has_tiles ? l : 0.f;
@@ -1047,8 +1077,7 @@ bool make_kv_map(CUtensorMap* map, const void* base, const pvlm_attn_params& p, 
 
 template <int NRP>
 constexpr int tc_smem_bytes() {
-  return 1024 /*alignment slack*/ + (kKStages + kVStages) * kTileBytes + 2 * NRP * 128 + 2 * NRP * 256 + 3 * 256 * 4 +
-         1024 * 4 + 32 * 8 + 64;
+  return 1024 /*alignment slack*/ + ring_slots(NRP) * kTileBytes + 2 * NRP * 128 + 2 * NRP * 256 + 3 * 256 * 4 + 32 * 8 + 64;
 }
 
 template <int NRP>
