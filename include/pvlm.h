@@ -271,6 +271,66 @@ typedef struct {
 pvlm_status pvlm_verify_step(const pvlm_step_params *p, void *stream);
 
 /* ------------------------------------------------------------------------
+ * Parallel decoding: the Pre-verify / Post-verify round loop on two streams.
+ *
+ * Stage II of the paper (Sec. 4.2 "Parallel Decoding"; Algorithm 1 and the
+ * appendix "Parallel Pipeline Details"): in every round the target verifies
+ * while the draft model writes `gamma` further tokens, each on its own
+ * stream; a rejection commits the replacement token, drops every other draft
+ * (the draft cache rolls back to the committed prefix) and returns to
+ * Pre-verify.
+ *   Pre-verify round : the draft writes d_0..d_{gamma-1}; d_0 alone is tested.
+ *                      accepted -> d_0 committed, gamma-1 drafts stay pending,
+ *                      next round is Post-verify; rejected -> replacement
+ *                      committed, drafts dropped.
+ *   Post-verify round: all pending drafts are tested in one batch while the
+ *                      draft writes gamma more behind them.  All accepted ->
+ *                      committed, the new gamma drafts become pending (no
+ *                      bonus token); else accepted prefix + replacement
+ *                      committed, everything else dropped, next is Pre-verify.
+ * The two models are stood in for by logit tables: row i of target_logits /
+ * draft_logits is that model's distribution for generated position i.  Each
+ * round runs, on `draft_stream`, the gamma draws from the draft rows
+ * (pvlm_spec_accept with gamma = 0, batch = gamma) and, on `target_stream`,
+ * the accept / reject / resample kernels over the tokens under test; if
+ * target_attn / draft_attn are given, the round also runs that attention
+ * call once on the target stream and gamma times on the draft stream as the
+ * forwards' memory traffic (their outputs are not used).  Random numbers are
+ * indexed by round: u_draft[r][s] draws the s-th token drafted in round r,
+ * u_accept[r][s] tests the s-th token verified in round r, u_resample[r]
+ * draws round r's replacement.
+ *
+ * The call is synchronous: it returns after K tokens have been committed
+ * (both streams idle).  tokens, round_log, n_rounds, round_ms are HOST
+ * pointers; everything else in the block is a DEVICE pointer.  Errors: bad
+ * sizes or NULL pointers PVLM_ERR_INVALID_ARG; P < K + 2*gamma + 1 or
+ * max_rounds exhausted PVLM_ERR_TOO_LARGE; workspace as for the other calls.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+  const float *target_logits, *draft_logits;  /* fp32 [P][row_stride], first V of a row used */
+  long long row_stride;                       /* elements, >= V                              */
+  int P, V, gamma, K;                         /* 1 <= gamma <= 64; K tokens to generate       */
+  float temperature;
+  const float *u_draft, *u_accept;            /* fp32 [max_rounds][gamma] in [0,1)            */
+  const float *u_resample;                    /* fp32 [max_rounds]                            */
+  int max_rounds;                             /* K rounds always suffice                      */
+  int *tokens;                                /* HOST int32 [K] out                           */
+  int *round_log;                             /* HOST int32 [max_rounds][6] out, nullable:
+                                                 mode (0 Pre, 1 Post), verified, accepted, committed, dropped, start */
+  int *n_rounds;                              /* HOST int32 out, nullable                     */
+  float *round_ms;                            /* HOST fp32 [max_rounds] out, nullable: device time of each round  */
+  const pvlm_attn_params *target_attn;        /* HOST pointer to a complete block, nullable   */
+  const pvlm_attn_params *draft_attn;         /* HOST pointer to a complete block, nullable   */
+  int serial;                                 /* 1 = vanilla SD order for comparison: the draft's work, then the
+                                                 target's, on target_stream only (same tokens)                */
+  void *workspace;
+  size_t workspace_bytes;
+} pvlm_decode_params;
+
+size_t pvlm_parallel_decode_workspace_bytes(const pvlm_decode_params *p);
+pvlm_status pvlm_parallel_decode(const pvlm_decode_params *p, void *target_stream, void *draft_stream);
+
+/* ------------------------------------------------------------------------
  * Draft window size from measured forward times (host arithmetic, no GPU).
  *
  * The window equals the pruned speed ratio c* = T_p / T_q(alpha) (paper

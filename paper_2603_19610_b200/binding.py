@@ -83,11 +83,21 @@ class StepParams(C.Structure):
                 ("copy_stream", C.c_void_p), ("event_a", C.c_void_p), ("event_b", C.c_void_p)]
 
 
+class DecodeParams(C.Structure):
+    _fields_ = [("target_logits", C.c_void_p), ("draft_logits", C.c_void_p), ("row_stride", C.c_longlong),
+                ("P", C.c_int), ("V", C.c_int), ("gamma", C.c_int), ("K", C.c_int), ("temperature", C.c_float),
+                ("u_draft", C.c_void_p), ("u_accept", C.c_void_p), ("u_resample", C.c_void_p), ("max_rounds", C.c_int),
+                ("tokens", C.c_void_p), ("round_log", C.c_void_p), ("n_rounds", C.c_void_p), ("round_ms", C.c_void_p),
+                ("target_attn", C.POINTER(AttnParams)), ("draft_attn", C.POINTER(AttnParams)), ("serial", C.c_int),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
 EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
            "pvlm_verify_attn_workspace_bytes", "pvlm_verify_attn", "pvlm_verify_attn_check",
            "pvlm_uvprune_workspace_bytes", "pvlm_uvprune_select_gather",
            "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept", "pvlm_verify_step",
-           "pvlm_uvprune_select_static", "pvlm_uvprune_similarity_workspace_bytes", "pvlm_uvprune_similarity", "pvlm_window_size")
+           "pvlm_uvprune_select_static", "pvlm_uvprune_similarity_workspace_bytes", "pvlm_uvprune_similarity", "pvlm_window_size",
+           "pvlm_parallel_decode_workspace_bytes", "pvlm_parallel_decode")
 
 
 def lib() -> C.CDLL:
@@ -115,6 +125,10 @@ def lib() -> C.CDLL:
             L.pvlm_uvprune_similarity_workspace_bytes.argtypes = [C.POINTER(SimilarityParams)]
             L.pvlm_uvprune_similarity.restype = C.c_int
             L.pvlm_uvprune_similarity.argtypes = [C.POINTER(SimilarityParams), C.c_void_p]
+            L.pvlm_parallel_decode_workspace_bytes.restype = C.c_size_t
+            L.pvlm_parallel_decode_workspace_bytes.argtypes = [C.POINTER(DecodeParams)]
+            L.pvlm_parallel_decode.restype = C.c_int
+            L.pvlm_parallel_decode.argtypes = [C.POINTER(DecodeParams), C.c_void_p, C.c_void_p]
             L.pvlm_uvprune_select_static.restype = C.c_int
             L.pvlm_uvprune_select_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                                      C.c_void_p, C.c_void_p, C.c_void_p]
@@ -410,3 +424,56 @@ def window_size(t_target: float, t_draft: float, mode: str = "nearest") -> int:
     f.restype = C.c_int
     f.argtypes = [C.c_double, C.c_double, C.c_int]
     return int(f(float(t_target), float(t_draft), {"nearest": 0, "down": 1, "up": 2}[mode]))
+
+
+def parallel_decode(target_logits, draft_logits, gamma: int, K: int, u_draft, u_accept, u_resample, *,
+                    temperature: float = 1.0, target_attn=None, draft_attn=None, serial: bool = False,
+                    draft_stream=None, want_ms: bool = False):
+    """The Pre-/Post-verify round loop on two streams (see pvlm_parallel_decode).
+    target_logits / draft_logits fp32 [P, V] on the device (row i = distribution of generated position i),
+    u_draft / u_accept fp32 [rounds, gamma], u_resample fp32 [rounds] on the device.  target_attn / draft_attn:
+    optional AttnParams blocks run as the forwards' traffic.  The target side uses the current stream.
+    Returns dict(tokens int32 [K], rounds, log int32 [rounds, 6], round_ms or None)."""
+    _need_cuda(target_logits, draft_logits, u_draft, u_accept, u_resample)
+    P, V = target_logits.shape
+    assert draft_logits.shape == (P, V) and target_logits.stride(1) == 1 and draft_logits.stride(0) == target_logits.stride(0)
+    assert target_logits.dtype == torch.float32 and draft_logits.dtype == torch.float32
+    dev = target_logits.device
+    max_rounds = u_resample.numel()
+    assert u_draft.shape == (max_rounds, gamma) and u_accept.shape == (max_rounds, gamma)
+    ud, ua, ur = u_draft.contiguous(), u_accept.contiguous(), u_resample.contiguous()
+    tokens = torch.empty(K, dtype=torch.int32)
+    log = torch.zeros((max_rounds, 6), dtype=torch.int32)
+    n_rounds = torch.zeros(1, dtype=torch.int32)
+    ms = torch.zeros(max_rounds, dtype=torch.float32) if want_ms else None
+    p = DecodeParams()
+    p.target_logits, p.draft_logits, p.row_stride = _ptr(target_logits), _ptr(draft_logits), target_logits.stride(0)
+    p.P, p.V, p.gamma, p.K, p.temperature = P, V, gamma, K, float(temperature)
+    p.u_draft, p.u_accept, p.u_resample, p.max_rounds = _ptr(ud), _ptr(ua), _ptr(ur), max_rounds
+    p.tokens, p.round_log, p.n_rounds = _ptr(tokens), _ptr(log), _ptr(n_rounds)
+    p.round_ms = _ptr(ms)
+    if target_attn is not None:
+        p.target_attn = C.pointer(target_attn)
+    if draft_attn is not None:
+        p.draft_attn = C.pointer(draft_attn)
+    p.serial = 1 if serial else 0
+    need = lib().pvlm_parallel_decode_workspace_bytes(C.byref(p))
+    ws = _workspace(dev, "decode", need)
+    p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()
+    if draft_stream is None and not serial:
+        draft_stream = _side_stream(dev)
+    st = lib().pvlm_parallel_decode(C.byref(p), _stream(dev), None if serial else C.c_void_p(draft_stream.cuda_stream))
+    if st != 0:
+        raise PvlmError(st, "pvlm_parallel_decode")
+    n = int(n_rounds[0])
+    return dict(tokens=tokens, rounds=n, log=log[:n], round_ms=None if ms is None else ms[:n])
+
+
+_SIDE: dict = {}
+
+
+def _side_stream(dev):
+    s = _SIDE.get(dev.index)
+    if s is None:
+        s = _SIDE[dev.index] = torch.cuda.Stream(device=dev)
+    return s

@@ -1,0 +1,74 @@
+"""Parity of pvlm_parallel_decode (Algorithm 1 on two streams) with the pipeline oracle: committed tokens and
+the per-round log (mode, verified, accepted, committed, dropped, start) must be identical."""
+import numpy as np
+import pytest
+import torch
+
+from oracle.pipeline import parallel_decode as oracle_decode
+from paper_2603_19610_b200 import binding, workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def make_case(V, K, gamma, sigma, seed):
+    rng = np.random.default_rng(seed)
+    P = K + 2 * gamma + 1
+    tl = (1.5 * rng.standard_normal((P, V))).astype(np.float32)
+    dl = (tl + sigma * rng.standard_normal((P, V))).astype(np.float32)
+    g = np.random.Generator(np.random.Philox(key=seed + 1000))
+    ud, ua, ur = wl.unit_uniforms(g, (K, gamma)), wl.unit_uniforms(g, (K, gamma)), wl.unit_uniforms(g, K)
+    return tl, dl, ud, ua, ur
+
+
+def gpu_decode(tl, dl, gamma, K, ud, ua, ur, **kw):
+    d = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return binding.parallel_decode(d(tl), d(dl), gamma, K, d(ud), d(ua), d(ur), **kw)
+
+
+def log_rows(log):
+    return [[r["mode"], r["verified"], r["accepted"], r["emitted"], r["dropped"], r["start"]] for r in log]
+
+
+@pytest.mark.parametrize("V,K,gamma,sigma,seed", [(50, 40, 4, 0.8, 3), (1000, 64, 9, 0.5, 7), (4099, 33, 1, 0.7, 11),
+                                                   (32000, 24, 5, 0.3, 5), (17, 80, 12, 1.5, 9), (152064, 12, 3, 0.4, 2)])
+def test_tokens_and_round_log_match_the_oracle(V, K, gamma, sigma, seed):
+    tl, dl, ud, ua, ur = make_case(V, K, gamma, sigma, seed)
+    ref = oracle_decode(tl, dl, gamma, K, ud, ua, ur)
+    out = gpu_decode(tl, dl, gamma, K, ud, ua, ur)
+    assert out["rounds"] == ref["rounds"]
+    assert out["log"].tolist() == log_rows(ref["log"])
+    np.testing.assert_array_equal(out["tokens"].numpy(), ref["tokens"])
+
+
+def test_serial_order_and_attention_payloads_do_not_change_the_tokens():
+    V, K, gamma = 2000, 48, 6
+    tl, dl, ud, ua, ur = make_case(V, K, gamma, 0.6, 21)
+    ref = oracle_decode(tl, dl, gamma, K, ud, ua, ur)
+    ser = gpu_decode(tl, dl, gamma, K, ud, ua, ur, serial=True)
+    np.testing.assert_array_equal(ser["tokens"].numpy(), ref["tokens"])
+    # forwards' traffic: a target verification over a 3000-token context and a draft decode step over 400 tokens
+    dev = torch.device("cuda")
+    mk = lambda *s: torch.randn(s, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    R = gamma + 1
+    qt, kt, vt = mk(2, R, 8, 128), mk(2, 3000 + R, 2, 128), mk(2, 3000 + R, 2, 128)
+    qd, kd, vd = mk(2, 1, 8, 128), mk(2, 401, 2, 128), mk(2, 401, 2, 128)
+    ws_t = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
+    ws_d = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
+    pt = binding.attn_params(qt, kt, vt, 3000, torch.empty_like(qt), None, None, workspace=ws_t)
+    pd = binding.attn_params(qd, kd, vd, 400, torch.empty_like(qd), None, None, workspace=ws_d)
+    out = gpu_decode(tl, dl, gamma, K, ud, ua, ur, target_attn=pt, draft_attn=pd, want_ms=True)
+    np.testing.assert_array_equal(out["tokens"].numpy(), ref["tokens"])
+    assert out["log"].tolist() == log_rows(ref["log"])
+    assert out["round_ms"].shape[0] == out["rounds"] and float(out["round_ms"].min()) > 0.0
+    assert binding.lib().pvlm_verify_attn_check(binding.C.byref(pt), None) == 0
+
+
+def test_argument_errors():
+    V, K, gamma = 64, 8, 3
+    tl, dl, ud, ua, ur = make_case(V, K, gamma, 0.5, 1)
+    with pytest.raises(binding.PvlmError, match="TOO_LARGE"):
+        gpu_decode(tl[:K + gamma], dl[:K + gamma], gamma, K, ud, ua, ur)           # too few positions
+    with pytest.raises(binding.PvlmError, match="INVALID_ARG"):
+        gpu_decode(tl, dl, gamma, K, ud, ua, ur, draft_stream=torch.cuda.current_stream())   # needs two streams
+    with pytest.raises(binding.PvlmError, match="TOO_LARGE"):
+        gpu_decode(tl, dl, gamma, K, ud[:2], ua[:2], ur[:2])                       # round tables exhausted
