@@ -133,3 +133,21 @@ def spec_accept_trials(target_logits, draft_logits, draft_tokens, uniforms, temp
         last = int(np.flatnonzero(W[t] > 0)[-1])
         tok[sel] = np.where(j >= V, last, j)
     return n, tok
+
+
+def tokenwise_acceptance(target_logits, draft_logits, tokens, uniforms, temperature: float = 1.0):
+    """Token-wise speculative sampling of a given text (appendix "Tasks and Metrics": the acceptance
+    rate A of a saved output under the full-context target): token x_n, drawn by a model with
+    distribution q_n, is accepted iff u_n < p_n(x_n) / q_n(x_n), every position on its own.
+    target_logits, draft_logits fp32 [N, V]; tokens int [N]; uniforms fp32 [N].
+    Returns dict(accepted bool [N], p_tok, q_tok fp32 [N], rate = mean(accepted)).
+    Same strictness and precision as `spec_accept`: u * q32 < p32 in fp32."""
+    p = softmax64(np.asarray(target_logits, dtype=np.float32), temperature)
+    q = softmax64(np.asarray(draft_logits, dtype=np.float32), temperature)
+    x = np.asarray(tokens, dtype=np.int64)
+    n = np.arange(x.shape[0])
+    p_tok = p[n, x].astype(np.float32)
+    q_tok = q[n, x].astype(np.float32)
+    u = np.asarray(uniforms, dtype=np.float32)
+    accepted = (u * q_tok).astype(np.float32) < p_tok
+    return dict(accepted=accepted, p_tok=p_tok, q_tok=q_tok, rate=float(accepted.mean()) if x.size else 0.0)

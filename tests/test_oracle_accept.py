@@ -244,3 +244,31 @@ def test_gamma_zero_is_plain_sampling():
     r = spec_accept(tl, np.zeros((0, 50), np.float32), np.zeros(0, np.int32), np.array([0.37], np.float32))
     assert r["n_accept"] == 0 and r["out_tokens"].shape == (1,)
     assert r["out_tokens"][0] == inverse_cdf(softmax64(tl)[0], 0.37)
+
+
+def test_tokenwise_acceptance_pins():
+    """(1) position by position it is the gamma = 1 accept rule; (2) with tokens drawn from q the acceptance
+    frequency is sum_x min(p, q) = 1 - TV(p, q); (3) identical models accept everything, a token outside the
+    target's support is rejected."""
+    from oracle.accept import tokenwise_acceptance
+    rng = np.random.default_rng(17)
+    N, V = 40, 37
+    tl = (1.5 * rng.standard_normal((N, V))).astype(np.float32)
+    dl = (tl + rng.standard_normal((N, V))).astype(np.float32)
+    x = wl.gumbel_draft_tokens(dl, rng)
+    u = wl.unit_uniforms(rng, N)
+    out = tokenwise_acceptance(tl, dl, x, u)
+    for n in range(N):
+        one = spec_accept(np.stack([tl[n], tl[n]]), dl[n][None], x[n:n + 1], np.array([u[n], 0.5], np.float32))
+        assert int(one["n_accept"]) == int(out["accepted"][n])
+        assert one["p_tok"][0] == out["p_tok"][n] and one["q_tok"][0] == out["q_tok"][n]
+    B = 200_000
+    g = np.random.Generator(np.random.Philox(key=5))
+    xs = wl.gumbel_draft_tokens(np.repeat(dl[:1], B, axis=0), g)
+    rate = tokenwise_acceptance(np.repeat(tl[:1], B, axis=0), np.repeat(dl[:1], B, axis=0), xs, wl.unit_uniforms(g, B))["rate"]
+    want = np.minimum(softmax64(tl[:1]), softmax64(dl[:1])).sum()
+    assert abs(rate - want) < 4 * np.sqrt(want * (1 - want) / B), (rate, want)
+    assert tokenwise_acceptance(tl, tl, x, u)["accepted"].all()
+    tl2 = tl.copy()
+    tl2[np.arange(N), x] = -np.inf
+    assert not tokenwise_acceptance(tl2, dl, x, u)["accepted"].any()
