@@ -293,6 +293,7 @@ def run_ours(args):
     if world == 1 and not args.no_draft_stream:
         draft_report = draft_stream_leg(cfg, dev, torch, binding, wl, Q, K, V, O, lse, mass, w, pp, pc, args)
         decode_report = decode_pipeline_leg(cfg, dev, torch, binding, Q, K, V, O, args)
+        rate_report = acceptance_rate_leg(cfg, dev, torch, binding)
 
     total_ms, e2e_ms = max_over_ranks(dist, torch, [total_ms, e2e_ms], dev)
 
@@ -340,6 +341,7 @@ def run_ours(args):
     if draft_report is not None:
         out["draft_stream"] = draft_report
         out["decode_pipeline"] = decode_report
+        out["acceptance_rate"] = rate_report
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, w)
     print(json.dumps(out))
@@ -406,6 +408,31 @@ def draft_stream_leg(cfg, dev, torch, binding, wl, Q, K, V, O, lse, mass, w, pp,
             "verify_step_us_alone": v_alone, "draft_window_us_alone": d_alone,
             "verify_step_us_concurrent": v_con, "draft_window_us_concurrent": d_con,
             "both_us_concurrent": max(v_con, d_con), "both_us_serial": v_alone + d_alone}
+
+
+def acceptance_rate_leg(cfg, dev, torch, binding, n_tok=1024):
+    """Token-wise acceptance of a 1024-token text under the config's vocabulary (pvlm_acceptance_rate): the
+    bandwidth-bound form of the vocab softmax, 8 * N * V bytes per call."""
+    g = torch.Generator(device=dev)
+    g.manual_seed(5)
+    tl = 1.5 * torch.randn((n_tok, cfg.V), generator=g, device=dev, dtype=torch.float32)
+    dl = tl + cfg.draft_sigma * torch.randn((n_tok, cfg.V), generator=g, device=dev, dtype=torch.float32)
+    x = torch.randint(0, cfg.V, (n_tok,), generator=g, device=dev, dtype=torch.int32)
+    u = torch.rand(n_tok, generator=g, device=dev)
+    for _ in range(3):
+        binding.acceptance_rate(tl, dl, x, u, want_probs=False)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 20
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        out = binding.acceptance_rate(tl, dl, x, u, want_probs=False)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    byts = 2 * n_tok * cfg.V * 4
+    return {"tokens": n_tok, "vocab": cfg.V, "us": ms * 1e3, "bytes": byts, "gbs": byts / ms / 1e6,
+            "accepted": int(out["n_accepted"].item())}
 
 
 def decode_pipeline_leg(cfg, dev, torch, binding, Q, K, V, O, args):

@@ -271,6 +271,39 @@ typedef struct {
 pvlm_status pvlm_verify_step(const pvlm_step_params *p, void *stream);
 
 /* ------------------------------------------------------------------------
+ * Token-wise acceptance rate of a given text (the paper's metric A).
+ *
+ * Appendix "Tasks and Metrics": the text a pruned model wrote is scored by
+ * token-wise speculative sampling under the full-context target: token x_n,
+ * whose writer had distribution q_n, counts as accepted iff
+ * u_n < p_n(x_n) / q_n(x_n) (evaluated as u_n * q32 < p32 in fp32, like
+ * pvlm_spec_accept), every position on its own, and A = accepted / N.
+ * One pass over the 2N logit rows (8 N V bytes): the bandwidth-bound form of
+ * the vocab softmax.
+ *
+ * All pointers are DEVICE pointers.  accepted / p_tok / q_tok hold one value
+ * per token; *n_accepted receives the count (the call zeroes it first).
+ * Tokens outside [0, V) count as rejected with p = 0, q = 1.  N = 0 is a
+ * no-op that writes *n_accepted = 0.  Supported: 0 <= N < 2^30, 1 <= V < 2^31.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+  const float *target_logits, *draft_logits;   /* fp32 [N][row stride], first V of a row used */
+  long long target_row_stride, draft_row_stride;
+  const int *tokens;                           /* int32 [N]                                   */
+  const float *uniforms;                       /* fp32 [N] in [0,1)                           */
+  int N, V;
+  float temperature;                           /* 0 or 1 => 1                                 */
+  int *accepted;                               /* int32 [N] out: 1 / 0                        */
+  float *p_tok, *q_tok;                        /* fp32 [N] out, nullable                      */
+  int *n_accepted;                             /* int32 [1] out                               */
+  void *workspace;
+  size_t workspace_bytes;
+} pvlm_rate_params;
+
+size_t pvlm_acceptance_rate_workspace_bytes(const pvlm_rate_params *p);
+pvlm_status pvlm_acceptance_rate(const pvlm_rate_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
  * Parallel decoding: the Pre-verify / Post-verify round loop on two streams.
  *
  * Stage II of the paper (Sec. 4.2 "Parallel Decoding"; Algorithm 1 and the

@@ -92,12 +92,21 @@ class DecodeParams(C.Structure):
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
+class RateParams(C.Structure):
+    _fields_ = [("target_logits", C.c_void_p), ("draft_logits", C.c_void_p),
+                ("target_row_stride", C.c_longlong), ("draft_row_stride", C.c_longlong),
+                ("tokens", C.c_void_p), ("uniforms", C.c_void_p), ("N", C.c_int), ("V", C.c_int),
+                ("temperature", C.c_float), ("accepted", C.c_void_p), ("p_tok", C.c_void_p), ("q_tok", C.c_void_p),
+                ("n_accepted", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
 EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
            "pvlm_verify_attn_workspace_bytes", "pvlm_verify_attn", "pvlm_verify_attn_check",
            "pvlm_uvprune_workspace_bytes", "pvlm_uvprune_select_gather",
            "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept", "pvlm_verify_step",
            "pvlm_uvprune_select_static", "pvlm_uvprune_similarity_workspace_bytes", "pvlm_uvprune_similarity", "pvlm_window_size",
-           "pvlm_parallel_decode_workspace_bytes", "pvlm_parallel_decode")
+           "pvlm_parallel_decode_workspace_bytes", "pvlm_parallel_decode",
+           "pvlm_acceptance_rate_workspace_bytes", "pvlm_acceptance_rate")
 
 
 def lib() -> C.CDLL:
@@ -129,6 +138,10 @@ def lib() -> C.CDLL:
             L.pvlm_parallel_decode_workspace_bytes.argtypes = [C.POINTER(DecodeParams)]
             L.pvlm_parallel_decode.restype = C.c_int
             L.pvlm_parallel_decode.argtypes = [C.POINTER(DecodeParams), C.c_void_p, C.c_void_p]
+            L.pvlm_acceptance_rate_workspace_bytes.restype = C.c_size_t
+            L.pvlm_acceptance_rate_workspace_bytes.argtypes = [C.POINTER(RateParams)]
+            L.pvlm_acceptance_rate.restype = C.c_int
+            L.pvlm_acceptance_rate.argtypes = [C.POINTER(RateParams), C.c_void_p]
             L.pvlm_uvprune_select_static.restype = C.c_int
             L.pvlm_uvprune_select_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                                      C.c_void_p, C.c_void_p, C.c_void_p]
@@ -477,3 +490,31 @@ def _side_stream(dev):
     if s is None:
         s = _SIDE[dev.index] = torch.cuda.Stream(device=dev)
     return s
+
+
+def acceptance_rate(target_logits, draft_logits, tokens, uniforms, temperature: float = 1.0, *, want_probs: bool = True):
+    """Token-wise acceptance of a given text (see pvlm_acceptance_rate).  target_logits / draft_logits fp32 [N, V],
+    tokens int32 [N], uniforms fp32 [N].  Returns dict(accepted int32 [N], n_accepted int32 [1], p_tok, q_tok)."""
+    _need_cuda(target_logits, draft_logits, tokens, uniforms)
+    N, V = target_logits.shape
+    assert draft_logits.shape == (N, V) and target_logits.dtype == torch.float32 and draft_logits.dtype == torch.float32
+    assert (N == 0 or (target_logits.stride(1) == 1 and draft_logits.stride(1) == 1)) and tokens.dtype == torch.int32
+    dev = target_logits.device
+    accepted = torch.empty(N, dtype=torch.int32, device=dev)
+    cnt = torch.empty(1, dtype=torch.int32, device=dev)
+    p_tok = torch.empty(N, dtype=torch.float32, device=dev) if want_probs else None
+    q_tok = torch.empty(N, dtype=torch.float32, device=dev) if want_probs else None
+    p = RateParams()
+    p.target_logits, p.draft_logits = _ptr(target_logits), _ptr(draft_logits)
+    p.target_row_stride = target_logits.stride(0) if N else V
+    p.draft_row_stride = draft_logits.stride(0) if N else V
+    p.tokens, p.uniforms = _ptr(tokens.contiguous()), _ptr(uniforms.contiguous())
+    p.N, p.V, p.temperature = N, V, float(temperature)
+    p.accepted, p.p_tok, p.q_tok, p.n_accepted = _ptr(accepted), _ptr(p_tok), _ptr(q_tok), _ptr(cnt)
+    need = lib().pvlm_acceptance_rate_workspace_bytes(C.byref(p))
+    ws = _workspace(dev, "rate", need)
+    p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()
+    st = lib().pvlm_acceptance_rate(C.byref(p), _stream(dev))
+    if st != 0:
+        raise PvlmError(st, "pvlm_acceptance_rate")
+    return dict(accepted=accepted, n_accepted=cnt, p_tok=p_tok, q_tok=q_tok)

@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libpvlm.so")
-SOURCES = ["pvlm_api.cu", "verify_attn.cu", "verify_attn_tc.cu", "uvprune.cu", "similarity.cu", "spec_accept.cu", "parallel_decode.cu"]
+SOURCES = ["pvlm_api.cu", "verify_attn.cu", "verify_attn_tc.cu", "uvprune.cu", "similarity.cu", "spec_accept.cu", "parallel_decode.cu", "acceptance_rate.cu"]
 
 
 def _nvcc() -> str:

@@ -36,7 +36,8 @@ def test_exports_every_declared_symbol():
 def test_header_is_c99_and_layouts_match():
     fields = {"pvlm_attn_params": binding.AttnParams, "pvlm_prune_params": binding.PruneParams,
               "pvlm_accept_params": binding.AcceptParams, "pvlm_step_params": binding.StepParams,
-              "pvlm_similarity_params": binding.SimilarityParams, "pvlm_decode_params": binding.DecodeParams}
+              "pvlm_similarity_params": binding.SimilarityParams, "pvlm_decode_params": binding.DecodeParams,
+              "pvlm_rate_params": binding.RateParams}
     prog = ['#include <stdio.h>', '#include <stddef.h>', '#include "pvlm.h"', 'int main(void){']
     for cname, st in fields.items():
         prog.append(f'printf("{cname} %zu\\n", sizeof({cname}));')
