@@ -261,10 +261,11 @@ typedef struct {
   const float *h_uniforms;
   void *h_o;
   int *h_n_accept, *h_out_tokens, *h_kept_idx;
-  /* Optional copy/compute overlap (all three NULL = everything on `stream`): a second cudaStream_t and two
-   * cudaEvent_t owned by the caller.  The accept inputs (logits, drafts, uniforms) are then uploaded on
-   * copy_stream while the attention runs, and o is downloaded on copy_stream while select/gather/accept
-   * run.  The call still orders everything so that synchronising `stream` alone is enough afterwards. */
+  /* Optional overlap (all three NULL = everything on `stream`): a second cudaStream_t and two cudaEvent_t
+   * owned by the caller.  The accept inputs (logits, drafts, uniforms) are then uploaded on copy_stream
+   * while the attention runs, the accept stage itself (which depends on nothing else in the step) runs on
+   * copy_stream behind them, and o is downloaded on copy_stream while select/gather run.  The call still
+   * orders everything so that synchronising `stream` alone is enough afterwards. */
   void *copy_stream, *event_a, *event_b;
 } pvlm_step_params;
 

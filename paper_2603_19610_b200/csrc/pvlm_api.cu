@@ -228,11 +228,22 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
       e = cudaMemcpyAsync(const_cast<int*>(c.draft_tokens), p->h_draft_tokens, B * c.gamma * 4, cudaMemcpyHostToDevice, cs);
     if (p->h_uniforms && ok())
       e = cudaMemcpyAsync(const_cast<float*>(c.uniforms), p->h_uniforms, B * (c.gamma + 1) * 4, cudaMemcpyHostToDevice, cs);
-    if (overlap && ok()) e = cudaEventRecord(ea, cs);           // accept inputs are on the device after this
   }
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   // ---- the three stages ----
   pvlm_status st;
+  // With a second stream the accept stage (which depends on nothing else in the step) runs there, right behind
+  // its uploads: its four small latency-bound kernels then overlap the attention's tail and the gather.
+  const bool accept_on_side = overlap && p->run_accept;
+  if (accept_on_side) {
+    if ((st = pvlm_spec_accept(&p->accept, cs)) != PVLM_OK) return st;
+    if (p->h_n_accept && ok())
+      e = cudaMemcpyAsync(p->h_n_accept, c.n_accept, (size_t)c.batch * 4, cudaMemcpyDeviceToHost, cs);
+    if (p->h_out_tokens && ok())
+      e = cudaMemcpyAsync(p->h_out_tokens, c.out_tokens, (size_t)c.batch * (c.gamma + 1) * 4, cudaMemcpyDeviceToHost, cs);
+    if (ok()) e = cudaEventRecord(ea, cs);                        // the accept stage and its results are complete after this
+    if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+  }
   if (p->run_attn && (st = pvlm_verify_attn(&p->attn, stream)) != PVLM_OK) return st;
   if (p->run_attn && p->h_o) {                                   // o is final: its download may overlap the rest
     const size_t q_layer = (size_t)a.R * a.Hq * a.D * 2;
@@ -245,17 +256,15 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   }
   if (p->run_prune && (st = pvlm_uvprune_select_gather(&p->prune, stream)) != PVLM_OK) return st;
-  if (p->run_accept) {
-    if (overlap && (e = cudaStreamWaitEvent(s, ea, 0)) != cudaSuccess) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
-    if ((st = pvlm_spec_accept(&p->accept, stream)) != PVLM_OK) return st;
-  }
+  if (p->run_accept && !accept_on_side && (st = pvlm_spec_accept(&p->accept, stream)) != PVLM_OK) return st;
   // ---- device -> host: the rest of this step's results ----
   if (p->run_prune && p->h_kept_idx && p->prune.k > 0 && ok())
     e = cudaMemcpyAsync(p->h_kept_idx, p->prune.kept_idx, (size_t)p->prune.k * 4, cudaMemcpyDeviceToHost, s);
-  if (p->run_accept && p->h_n_accept && ok())
+  if (p->run_accept && !accept_on_side && p->h_n_accept && ok())
     e = cudaMemcpyAsync(p->h_n_accept, c.n_accept, (size_t)c.batch * 4, cudaMemcpyDeviceToHost, s);
-  if (p->run_accept && p->h_out_tokens && ok())
+  if (p->run_accept && !accept_on_side && p->h_out_tokens && ok())
     e = cudaMemcpyAsync(p->h_out_tokens, c.out_tokens, (size_t)c.batch * (c.gamma + 1) * 4, cudaMemcpyDeviceToHost, s);
+  if (accept_on_side && ok()) e = cudaStreamWaitEvent(s, ea, 0);                     // `stream` now also covers the accept stage
   if (overlap && p->run_attn && p->h_o && ok()) e = cudaStreamWaitEvent(s, eb, 0);   // `stream` now also covers the o download
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   return PVLM_OK;
