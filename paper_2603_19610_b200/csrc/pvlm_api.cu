@@ -9,6 +9,14 @@ static thread_local int g_last_cuda_error = 0;
 
 void set_cuda_error(int e) { g_last_cuda_error = e; }
 
+static thread_local cudaEvent_t g_after_main_event = nullptr;
+void set_after_main_event(cudaEvent_t ev) { g_after_main_event = ev; }
+cudaEvent_t take_after_main_event() {
+  cudaEvent_t ev = g_after_main_event;
+  g_after_main_event = nullptr;
+  return ev;
+}
+
 pvlm_status check_launch() {
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
@@ -106,7 +114,7 @@ size_t pvlm_uvprune_workspace_bytes(const pvlm_prune_params* p) {
   return uvprune_workspace(*p);
 }
 
-pvlm_status pvlm_uvprune_select_gather(const pvlm_prune_params* p, void* stream) {
+static pvlm_status validate_prune(const pvlm_prune_params* p) {
   if (!p) return PVLM_ERR_INVALID_ARG;
   if (p->m < 0 || p->k < 0 || p->k > p->m || p->vis_start < 0) return PVLM_ERR_INVALID_ARG;
   if (p->m > (1 << 24)) return PVLM_ERR_UNSUPPORTED;
@@ -125,7 +133,11 @@ pvlm_status pvlm_uvprune_select_gather(const pvlm_prune_params* p, void* stream)
       if (p->dst_layer_stride_bytes < dst_len * p->row_bytes || p->dst_layer_stride_bytes % 16) return PVLM_ERR_INVALID_ARG;
     }
   }
-  const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, uvprune_workspace(*p));
+  return check_ws(p->workspace, p->workspace_bytes, uvprune_workspace(*p));
+}
+
+pvlm_status pvlm_uvprune_select_gather(const pvlm_prune_params* p, void* stream) {
+  const pvlm_status w = validate_prune(p);
   if (w != PVLM_OK) return w;
   return launch_uvprune(*p, (cudaStream_t)stream);
 }
@@ -231,20 +243,36 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
   }
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   // ---- the three stages ----
+  // With a second stream, what does not depend on the attention's results runs there: the accept stage and the
+  // part of the gather that does not depend on the selection (the rows before and after the visual span).  Both
+  // are queued behind an event that the attention records right after its main kernel, so they start when
+  // that kernel ends and fill the gap in which the main stream runs the small combine / mass / select kernels
+  // and HBM would otherwise idle (queued earlier they would only take SMs from the main kernel's start).
   pvlm_status st;
-  // With a second stream the accept stage (which depends on nothing else in the step) runs there, right behind
-  // its uploads: its four small latency-bound kernels then overlap the attention's tail and the gather.
   const bool accept_on_side = overlap && p->run_accept;
+  const bool split_gather = overlap && p->run_prune && p->prune.src_k;
+  if (split_gather && (st = validate_prune(&p->prune)) != PVLM_OK) return st;
+  if (p->run_attn) {
+    if (accept_on_side || split_gather) set_after_main_event(eb);
+    st = pvlm_verify_attn(&p->attn, stream);
+    const bool recorded = take_after_main_event() == nullptr;     // consumed by the launch => eb is recorded
+    if (st != PVLM_OK) return st;
+    if ((accept_on_side || split_gather) && !recorded) e = cudaEventRecord(eb, s);
+  } else if (accept_on_side || split_gather) {
+    e = cudaEventRecord(eb, s);
+  }
+  if ((accept_on_side || split_gather) && ok()) e = cudaStreamWaitEvent(cs, eb, 0);
+  if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+  if (split_gather && (st = launch_uvprune_parts(p->prune, false, 1, cs)) != PVLM_OK) return st;
   if (accept_on_side) {
     if ((st = pvlm_spec_accept(&p->accept, cs)) != PVLM_OK) return st;
     if (p->h_n_accept && ok())
       e = cudaMemcpyAsync(p->h_n_accept, c.n_accept, (size_t)c.batch * 4, cudaMemcpyDeviceToHost, cs);
     if (p->h_out_tokens && ok())
       e = cudaMemcpyAsync(p->h_out_tokens, c.out_tokens, (size_t)c.batch * (c.gamma + 1) * 4, cudaMemcpyDeviceToHost, cs);
-    if (ok()) e = cudaEventRecord(ea, cs);                        // the accept stage and its results are complete after this
-    if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   }
-  if (p->run_attn && (st = pvlm_verify_attn(&p->attn, stream)) != PVLM_OK) return st;
+  if ((accept_on_side || split_gather) && ok()) e = cudaEventRecord(ea, cs);   // the side stream's stages are complete after this
+  if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   if (p->run_attn && p->h_o) {                                   // o is final: its download may overlap the rest
     const size_t q_layer = (size_t)a.R * a.Hq * a.D * 2;
     if (overlap) {
@@ -255,7 +283,10 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     if (overlap && ok()) e = cudaEventRecord(eb, cs);
     if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   }
-  if (p->run_prune && (st = pvlm_uvprune_select_gather(&p->prune, stream)) != PVLM_OK) return st;
+  if (p->run_prune) {
+    st = split_gather ? launch_uvprune_parts(p->prune, true, 2, s) : pvlm_uvprune_select_gather(&p->prune, stream);
+    if (st != PVLM_OK) return st;
+  }
   if (p->run_accept && !accept_on_side && (st = pvlm_spec_accept(&p->accept, stream)) != PVLM_OK) return st;
   // ---- device -> host: the rest of this step's results ----
   if (p->run_prune && p->h_kept_idx && p->prune.k > 0 && ok())
@@ -264,7 +295,7 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     e = cudaMemcpyAsync(p->h_n_accept, c.n_accept, (size_t)c.batch * 4, cudaMemcpyDeviceToHost, s);
   if (p->run_accept && !accept_on_side && p->h_out_tokens && ok())
     e = cudaMemcpyAsync(p->h_out_tokens, c.out_tokens, (size_t)c.batch * (c.gamma + 1) * 4, cudaMemcpyDeviceToHost, s);
-  if (accept_on_side && ok()) e = cudaStreamWaitEvent(s, ea, 0);                     // `stream` now also covers the accept stage
+  if ((accept_on_side || split_gather) && ok()) e = cudaStreamWaitEvent(s, ea, 0);   // `stream` now also covers the side stream's stages
   if (overlap && p->run_attn && p->h_o && ok()) e = cudaStreamWaitEvent(s, eb, 0);   // `stream` now also covers the o download
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   return PVLM_OK;

@@ -19,6 +19,12 @@ inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 pvlm_status check_launch();
 void set_cuda_error(int e);
 
+// A cudaEvent_t that the next attention launch of this host thread records right after its main kernel
+// (before the combine / mass kernels).  take_* returns the pending event (nullptr once a launch has used it)
+// and clears it.
+void set_after_main_event(cudaEvent_t ev);
+cudaEvent_t take_after_main_event();
+
 // ---- verify attention -----------------------------------------------------
 constexpr int kAttnBN = 64;           // keys per tile
 
@@ -52,6 +58,7 @@ pvlm_status launch_verify_attn(const pvlm_attn_params& p, const AttnPlan& plan, 
 
 // ---- uvprune ----------------------------------------------------------------
 pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s);
+pvlm_status launch_uvprune_parts(const pvlm_prune_params& p, bool select, int part, cudaStream_t s);
 size_t uvprune_workspace(const pvlm_prune_params& p);
 
 // ---- similarity (hidden-state criterion) --------------------------------------------

@@ -385,6 +385,8 @@ struct GatherArgs {
   int4 *dst_k, *dst_v;
   const int* kept;
   int vis_start, m, k, dst_len, n_layers;
+  int seg0_lo, seg0_len, seg1_lo, seg1_len;   // the destination rows this launch writes: two runs, rows = their sum
+  int rows;
   int row_vec;                       // 16-byte units per row
   long long src_ls_vec, dst_ls_vec;  // layer strides in 16-byte units
 };
@@ -392,14 +394,15 @@ struct GatherArgs {
 // One thread moves 16 bytes of K and 16 bytes of V per step; a destination row
 // maps to its source row through the kept-index list.
 __global__ void __launch_bounds__(256) uvprune_gather_kernel(const GatherArgs a) {
-  const long long per_layer = (long long)a.dst_len * a.row_vec;
+  const long long per_layer = (long long)a.rows * a.row_vec;
   const long long total = per_layer * a.n_layers;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += stride) {
     const int layer = (int)(u / per_layer);
     const long long w = u - (long long)layer * per_layer;
-    const int drow = (int)(w / a.row_vec);
-    const int c = (int)(w - (long long)drow * a.row_vec);
+    const int r = (int)(w / a.row_vec);
+    const int c = (int)(w - (long long)r * a.row_vec);
+    const int drow = r < a.seg0_len ? a.seg0_lo + r : a.seg1_lo + (r - a.seg0_len);
     int srow;
     if (drow < a.vis_start) srow = drow;
     else if (drow < a.vis_start + a.k) srow = a.vis_start + __ldg(a.kept + (drow - a.vis_start));
@@ -417,7 +420,11 @@ __global__ void __launch_bounds__(256) uvprune_gather_kernel(const GatherArgs a)
 
 size_t uvprune_workspace(const pvlm_prune_params& p) { return align_up((size_t)(p.m > 0 ? p.m : 1) * 4, 256); }
 
-pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s) {
+pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s) { return launch_uvprune_parts(p, true, 0, s); }
+
+// part 0: all destination rows; 1: only the rows that do not depend on the selection (before and after the
+// visual span); 2: only the selected visual rows.
+pvlm_status launch_uvprune_parts(const pvlm_prune_params& p, bool select, int part, cudaStream_t s) {
   SelArgs sa;
   sa.cur = p.mass_cur + p.vis_start;
   sa.ref = p.mass_ref ? p.mass_ref + p.vis_start : nullptr;
@@ -426,7 +433,7 @@ pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s) {
   sa.kept = p.kept_idx;
   sa.m = p.m;
   sa.k = p.k;
-  if (p.m > 0) {
+  if (select && p.m > 0) {
     const char* impl = getenv("PVLM_SELECT_IMPL");       // "cta": single-CTA kernels only (second implementation for tests)
     const bool one_cta = impl && strcmp(impl, "cta") == 0;
     if (!one_cta && p.m <= kSelCluster * kSelThreads * 4) uvprune_select_cluster_kernel<4><<<kSelCluster, kSelThreads, 0, s>>>(sa);
@@ -448,10 +455,17 @@ pvlm_status launch_uvprune(const pvlm_prune_params& p, cudaStream_t s) {
     g.row_vec = (int)(p.row_bytes / 16);
     g.src_ls_vec = p.src_layer_stride_bytes / 16;
     g.dst_ls_vec = p.dst_layer_stride_bytes / 16;
-    const long long total = (long long)g.dst_len * g.row_vec * g.n_layers;
+    g.seg1_lo = g.seg1_len = 0;
+    if (part == 0) { g.seg0_lo = 0; g.seg0_len = g.dst_len; }
+    else if (part == 1) { g.seg0_lo = 0; g.seg0_len = p.vis_start; g.seg1_lo = p.vis_start + p.k; g.seg1_len = g.dst_len - g.seg1_lo; }
+    else { g.seg0_lo = p.vis_start; g.seg0_len = p.k; }
+    g.rows = g.seg0_len + g.seg1_len;
+    const long long total = (long long)g.rows * g.row_vec * g.n_layers;
     if (total > 0) {
       long long blocks = (total + 255) / 256;
-      const long long cap = (long long)kNumSMs * 16;
+      // Whole-gather launches loop inside a resident set of CTAs.  A partial launch runs beside latency-critical
+      // kernels of another stream, so its CTAs are kept short (two copies per thread): they give SM slots back quickly.
+      const long long cap = part == 0 ? (long long)kNumSMs * 16 : (blocks + 1) / 2;
       if (blocks > cap) blocks = cap;
       uvprune_gather_kernel<<<(int)blocks, 256, 0, s>>>(g);
     }

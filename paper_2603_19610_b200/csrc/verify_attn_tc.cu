@@ -1196,6 +1196,7 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
     default: return PVLM_ERR_UNSUPPORTED;
   }
   if (p.prof_event_end) cudaEventRecord((cudaEvent_t)p.prof_event_end, s);
+  if (cudaEvent_t ev = take_after_main_event()) cudaEventRecord(ev, s);     // lets a caller queue other work behind the main kernel
   CombineArgs c;
   c.part_o = a.part_o; c.part_ml = a.part_ml; c.o = (__nv_bfloat16*)p.o; c.lse = p.lse; c.lse2 = lse2;
   c.R = p.R; c.Hq = p.Hq; c.Hkv = p.Hkv; c.G = a.G; c.rows = a.rows; c.nrp = plan.nrp;
