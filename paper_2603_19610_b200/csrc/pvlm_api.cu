@@ -224,6 +224,11 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
                               cudaMemcpyHostToDevice, s);
     }
   }
+  if (overlap && p->run_attn && (p->h_q || p->h_k_window || p->h_v_window) && ok()) {
+    // the attention's own inputs go first over the link: the accept inputs, needed much later, queue behind them
+    e = cudaEventRecord(eb, s);
+    if (ok()) e = cudaStreamWaitEvent(cs, eb, 0);
+  }
   if (p->run_accept) {
     if (c.gamma < 0 || c.V < 1 || c.batch < 1) return PVLM_ERR_INVALID_ARG;
     if (p->h_target_logits || p->h_draft_logits) {
