@@ -128,6 +128,8 @@ def test_verify_step_host_buffers_config0():
     for host_t in h_out.values():
         host_t.zero_()
     tl2.zero_(); dl2.zero_(); q2.zero_(); o2.zero_()
+    dk2.zero_(); dv2.zero_(); kept2.zero_(); mass2.zero_()   # everything the step writes must be written again
+    outs["n_accept"].fill_(-7); outs["out_tokens"].fill_(-7)
     cs, ea, eb = torch.cuda.Stream(), torch.cuda.Event(), torch.cuda.Event()
     ea.record(); eb.record()
     torch.cuda.synchronize()
@@ -141,6 +143,31 @@ def test_verify_step_host_buffers_config0():
     assert torch.equal(dk2, dk_e) and torch.equal(dv2, dv_e)
     assert int(h_out["h_n_accept"]) == int(acc_e["n_accept"])
     assert torch.equal(h_out["h_out_tokens"], acc_e["out_tokens"].cpu())
+
+
+def test_verify_step_overlap_mode_splits_the_gather_correctly():
+    """Overlap mode copies the rows outside the visual span on the second stream and the selected rows on the
+    main stream: with rows before AND after the visual span the compacted caches must equal the one-call result."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(77)
+    L, S, Hkv, D, v0, m, k = 3, 1029, 4, 128, 5, 896, 224
+    src_k = torch.randn((L, S, Hkv, D), device=dev).to(torch.bfloat16)
+    src_v = torch.randn((L, S, Hkv, D), device=dev).to(torch.bfloat16)
+    cur = torch.from_numpy(rng.random(S).astype(np.float32)).to(dev)
+    ref = torch.from_numpy(rng.random(S).astype(np.float32)).to(dev)
+    kept_e, _, dk_e, dv_e = binding.uvprune_select_gather(cur, ref, v0, m, k, src_k, src_v)
+    kept = torch.zeros(k, dtype=torch.int32, device=dev)
+    dk = torch.zeros((L, S - m + k, Hkv, D), dtype=torch.bfloat16, device=dev)
+    dv = torch.zeros_like(dk)
+    pp = binding.prune_params(cur, ref, v0, m, k, kept, None, src_k, src_v, dk, dv)
+    cs, ea, eb = torch.cuda.Stream(), torch.cuda.Event(), torch.cuda.Event()
+    ea.record(); eb.record()
+    torch.cuda.synchronize()
+    for _ in range(2):                                            # twice: events and streams are reused across steps
+        dk.zero_(); dv.zero_(); kept.zero_()
+        binding.verify_step(None, pp, None, device=dev, overlap=(cs, ea, eb))
+        torch.cuda.current_stream().synchronize()
+        assert torch.equal(kept, kept_e) and torch.equal(dk, dk_e) and torch.equal(dv, dv_e)
 
 
 def test_draft_and_verify_streams_run_concurrently_and_agree():
