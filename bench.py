@@ -326,8 +326,8 @@ def run_ours(args):
     kern_ms = sum(main_kernel_ms) / len(main_kernel_ms)
     ab_kernel = L * (2 * T * cfg.Hkv * cfg.D * 2 + R * cfg.Hq * cfg.D * 2)      # K and V once, Q once; partials excluded
     achieved = ab_kernel / (kern_ms * 1e-3) / 1e9
-    # DRAM traffic of one launch of the dominant kernel, from the ncu capture summarised in
-    # profiles/attn_tc_kernel_cfg2_4layers.md: 544.96 MB (read + write) for 4 layers of the config-2
+    # DRAM traffic of one launch of the dominant kernel, from the ncu capture of that kernel summarised under
+    # profiles/: 544.96 MB (read + write) for 4 layers of the config-2
     # geometry, which grows in proportion to the layers processed.
     traffic = 544.96e6 / 4 * L if cfg.cid == 2 else None
     out = {
