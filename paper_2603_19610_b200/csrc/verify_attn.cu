@@ -413,7 +413,7 @@ bool make_attn_plan(const pvlm_attn_params& p, AttnPlan& plan) {
   }
   // main pass on the tcgen05 kernel whenever it applies (PVLM_ATTN_IMPL=mma forces the mma.sync kernel)
   const char* impl = getenv("PVLM_ATTN_IMPL");
-  plan.use_tc = (p.D == 128) && !(impl && strcmp(impl, "mma") == 0) && make_attn_tc_plan(p, plan.tc);
+  plan.use_tc = (p.D == 128 || p.D == 64) && !(impl && strcmp(impl, "mma") == 0) && make_attn_tc_plan(p, plan.tc);
   plan.off_tc = off;
   if (plan.use_tc) off += align_up(plan.tc.total, 256);
   plan.total = off;

@@ -1,4 +1,7 @@
-// Window-verify GQA attention on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), D = 128.
+// Window-verify GQA attention on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), D = 128 or 64.
+// (D = 64 runs the same kernels on channels padded to 128: the tensor map knows 64 channels, so the TMA
+// box of channels 64..127 is out of range and arrives as zeros without touching memory; Q's upper half stays
+// zero in shared memory; only the global reads of Q and the writes of O know the real row length.)
 //
 // Work decomposition ("stream-K"): the (layer, KV head) items are cut into 128-key tiles, the
 // flattened tile sequence is divided evenly among one persistent CTA per SM, and a CTA walks its
@@ -52,6 +55,7 @@ struct TcArgs {
   float *part_o, *part_ml;
   int* status;
   int R, Hq, Hkv, G, n_ctx, T, rows, n_layers;
+  int D;                     // real head dimension (64 or 128)
   long long q_ls;
   float scale_log2;
   int tiles_per_item;        // Tt
@@ -482,11 +486,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
         // ---- stage Q of this (layer, KV head) in the K-major 128B-swizzled layout ----
         {
-          const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * 128;
-          for (int idx = st; idx < a.rows * 16; idx += kSoftmaxThreads) {
-            const int row = idx >> 4, c = idx & 15;
+          const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * a.D;
+          const int cpr = a.D >> 3;                        // 16-byte pieces per query row: 16, or 8 when D = 64
+          for (int idx = st; idx < a.rows * cpr; idx += kSoftmaxThreads) {
+            const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
             const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
-            const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * 128 + c * 8);
+            const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
             *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val;
           }
           fence_proxy_async();
@@ -714,6 +719,7 @@ struct CombineArgs {
   __nv_bfloat16* o;
   float *lse, *lse2;
   int R, Hq, Hkv, G, rows, nrp, tiles_per_item, seg_max, n_cta;
+  int D;                     // real head dimension; partials are always 128 wide
   long long total_tiles, q_ls;
 };
 
@@ -765,8 +771,9 @@ __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs 
       }
       const float inv = 1.f / l;
       const int r = row / a.G, g = row - r * a.G;
-      __nv_bfloat16* dst = a.o + (long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * 128 + lane * 4;
-      *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(acc.x * inv, acc.y * inv), pack2(acc.z * inv, acc.w * inv));
+      __nv_bfloat16* dst = a.o + (long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * a.D + lane * 4;
+      if (lane * 4 < a.D)
+        *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(acc.x * inv, acc.y * inv), pack2(acc.z * inv, acc.w * inv));
       if (lane == 0) {
         const long long li = (long long)layer * a.Hq * a.R + (kvh * a.G + g) * a.R + r;
         const float v2 = mstar + log2f(l);
@@ -809,8 +816,9 @@ __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs 
     const float inv = 1.f / lt;
     const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
     const int r = row / a.G, g = row - r * a.G;
-    __nv_bfloat16* dst = a.o + (long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * 128 + lane * 4;
-    *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(t.x * inv, t.y * inv), pack2(t.z * inv, t.w * inv));
+    __nv_bfloat16* dst = a.o + (long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * a.D + lane * 4;
+    if (lane * 4 < a.D)
+      *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(t.x * inv, t.y * inv), pack2(t.z * inv, t.w * inv));
     if (lane == 0) {
       const long long li = (long long)layer * a.Hq * a.R + (kvh * a.G + g) * a.R + r;
       const float v2 = mstar + log2f(lt);
@@ -835,6 +843,7 @@ struct TcMassArgs {
   float* part_mass;          // [n_mass][Hkv][T_pad]
   int* status;
   int R, Hq, Hkv, G, n_ctx, T, T_pad, rows;
+  int D;                     // real head dimension (64 or 128)
   long long q_ls;
   float scale_log2;
   int tiles_per_item, n_cta;
@@ -950,11 +959,12 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
         const int zrow = item / a.Hkv, kvh = item - zrow * a.Hkv;
         const int layer = a.mass_listed ? a.mass_layer[zrow] : zrow;
         {
-          const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * 128;
-          for (int idx = st; idx < a.rows * 16; idx += kSoftmaxThreads) {
-            const int row = idx >> 4, c = idx & 15;
+          const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * a.D;
+          const int cpr = a.D >> 3;                        // 16-byte pieces per query row: 16, or 8 when D = 64
+          for (int idx = st; idx < a.rows * cpr; idx += kSoftmaxThreads) {
+            const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
             const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
-            const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * 128 + c * 8);
+            const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
             *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val;
           }
           if (st < 128) {
@@ -1065,7 +1075,7 @@ EncodeTiledFn encode_tiled_fn() {
 bool make_kv_map(CUtensorMap* map, const void* base, const pvlm_attn_params& p, int T) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
-  const cuuint64_t dims[4] = {128, (cuuint64_t)p.Hkv, (cuuint64_t)T, (cuuint64_t)p.n_layers};
+  const cuuint64_t dims[4] = {(cuuint64_t)p.D, (cuuint64_t)p.Hkv, (cuuint64_t)T, (cuuint64_t)p.n_layers};   // D = 64: box 1 is all fill
   const cuuint64_t layer_stride = p.n_layers > 1 ? (cuuint64_t)p.kv_layer_stride : (cuuint64_t)T * p.kv_token_stride;
   const cuuint64_t strides[3] = {(cuuint64_t)p.kv_head_stride * 2, (cuuint64_t)p.kv_token_stride * 2, layer_stride * 2};
   const cuuint32_t box[4] = {64, 1, (cuuint32_t)kTile, 1};
@@ -1109,6 +1119,7 @@ pvlm_status launch_attn_mass_tc(const pvlm_attn_params& p, const float* lse2, fl
   TcMassArgs a;
   a.q = (const __nv_bfloat16*)p.q; a.lse2 = lse2; a.part_mass = part_mass; a.status = status;
   a.R = p.R; a.Hq = p.Hq; a.Hkv = p.Hkv; a.G = G; a.n_ctx = p.n_ctx; a.T = T; a.T_pad = (int)align_up(T, kAttnBN); a.rows = rows;
+  a.D = p.D;
   a.q_ls = p.q_layer_stride;
   const float scale = (p.softmax_scale == 0.f) ? 1.0f / sqrtf((float)p.D) : p.softmax_scale;
   a.scale_log2 = scale * kLog2e;
@@ -1136,7 +1147,7 @@ pvlm_status launch_attn_mass_tc(const pvlm_attn_params& p, const float* lse2, fl
 }
 
 bool make_attn_tc_plan(const pvlm_attn_params& p, AttnTcPlan& plan) {
-  if (p.D != 128 || p.Hkv <= 0 || p.Hq % p.Hkv != 0) return false;
+  if ((p.D != 128 && p.D != 64) || p.Hkv <= 0 || p.Hq % p.Hkv != 0) return false;
   const int G = p.Hq / p.Hkv;
   const int rows = G * p.R;
   if (rows > 96) return false;                   // wider groups stay on the mma.sync kernel
@@ -1171,6 +1182,7 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   a.status = (int*)(ws + plan.off_status);
   a.R = p.R; a.Hq = p.Hq; a.Hkv = p.Hkv; a.G = p.Hq / p.Hkv; a.n_ctx = p.n_ctx; a.T = plan.T;
   a.rows = a.G * p.R; a.n_layers = p.n_layers;
+  a.D = p.D;
   a.q_ls = p.q_layer_stride;
   const float scale = (p.softmax_scale == 0.f) ? 1.0f / sqrtf((float)p.D) : p.softmax_scale;
   a.scale_log2 = scale * kLog2e;
@@ -1202,6 +1214,7 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   c.R = p.R; c.Hq = p.Hq; c.Hkv = p.Hkv; c.G = a.G; c.rows = a.rows; c.nrp = plan.nrp;
   c.tiles_per_item = plan.tiles_per_item; c.seg_max = plan.seg_max; c.n_cta = plan.n_cta;
   c.total_tiles = plan.total_tiles; c.q_ls = p.q_layer_stride;
+  c.D = p.D;
   {
     const int items = p.Hkv * p.n_layers;
     int rows_y = 2048 / items;                            // enough blocks to fill the GPU, not tens of thousands

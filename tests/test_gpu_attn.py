@@ -163,9 +163,28 @@ def test_tensor_core_path_rescales_inside_long_runs(monkeypatch):
 def test_mma_sync_path_still_matches(monkeypatch):
     """PVLM_ATTN_IMPL=mma forces the mma.sync kernel for D = 128 as well (the second implementation)."""
     monkeypatch.setenv("PVLM_ATTN_IMPL", "mma")
-    for (Hq, Hkv, D, n_ctx, R) in [(40, 8, 128, 2500, 13), (28, 4, 128, 1000, 9)]:
+    for (Hq, Hkv, D, n_ctx, R) in [(40, 8, 128, 2500, 13), (28, 4, 128, 1000, 9), (6, 2, 64, 700, 5), (14, 2, 64, 70, 1)]:
         qb, kb, vb = wl.make_qkv(Hq, Hkv, D, R, n_ctx + R, sink=True, seed=9 + n_ctx)
         run_case(qb, kb, vb, n_ctx)
+
+
+def test_head_dim_64_on_the_tensor_core_path(monkeypatch):
+    """D = 64 runs the tcgen05 kernels on channels padded to 128 by the TMA's out-of-range fill: several layers,
+    long tile runs on few CTAs (many segments per CTA), batched launch with mass rows."""
+    monkeypatch.setenv("PVLM_TC_CTAS", "5")
+    L, Hq, Hkv, D, n_ctx, R = 3, 14, 2, 64, 1500, 4
+    layers = [wl.make_qkv(Hq, Hkv, D, R, n_ctx + R, sink=True, seed=300 + l) for l in range(L)]
+    q = torch.stack([bf16_cuda(x[0]) for x in layers])
+    k = torch.stack([bf16_cuda(x[1]) for x in layers])
+    v = torch.stack([bf16_cuda(x[2]) for x in layers])
+    o, lse, mass = binding.verify_attn(q, k, v, n_ctx, want_mass=True, mass_layers=[0, 2], check=True)
+    for i, l in enumerate([0, 2]):
+        O, Lr, M = oracle_attn(*layers[l], n_ctx)
+        assert_o_close(o[l], O)
+        assert_rel_close(lse[l].cpu().numpy(), Lr, 1e-4, "lse")
+        assert_rel_close(mass[i].cpu().numpy(), M, 1e-4, "mass")
+    O1, L1, _ = oracle_attn(*layers[1], n_ctx)
+    assert_o_close(o[1], O1)
 
 
 def test_head_major_cache_layout():
