@@ -227,7 +227,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
 // ---------------------------------------------------------------------------------------------
 // K and V tiles share one ring of 32 KB slots, filled and drained in the order the issuer consumes them.
 // Five slots fit beside Q and the two P buffers up to 80 padded rows.
-__host__ __device__ constexpr int ring_slots(int nrp) { return nrp <= 80 ? 5 : 4; }
+__host__ __device__ constexpr int ring_slots(int nrp) { return nrp <= 80 ? 5 : nrp <= 112 ? 4 : 3; }
 __host__ __device__ constexpr int s_bufs(int nrp) { return (512 - 2 * nrp) / nrp >= 4 ? 4 : (512 - 2 * nrp) / nrp; }
 
 // HT: the last 16-column chunk holds at most 8 real query rows, so only its first 8 columns are processed.
@@ -244,7 +244,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   constexpr uint32_t TMEM_COLS = NEED <= 32 ? 32 : NEED <= 64 ? 64 : NEED <= 128 ? 128 : NEED <= 256 ? 256 : 512;
   constexpr uint32_t IDESC_QK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NRP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   constexpr uint32_t IDESC_PV = IDESC_QK | (1u << 15) | (1u << 16);
-  static_assert(NRP % 16 == 0 && NRP <= 96 && NSB >= 2, "row padding");
+  static_assert(NRP % 16 == 0 && NRP <= 128 && NSB >= 2, "row padding");
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -1150,7 +1150,7 @@ bool make_attn_tc_plan(const pvlm_attn_params& p, AttnTcPlan& plan) {
   if ((p.D != 128 && p.D != 64) || p.Hkv <= 0 || p.Hq % p.Hkv != 0) return false;
   const int G = p.Hq / p.Hkv;
   const int rows = G * p.R;
-  if (rows > 96) return false;                   // wider groups stay on the mma.sync kernel
+  if (rows > 128) return false;                  // one tile row per TMEM lane: at most 128 query rows per KV head
   plan.nrp = (rows + 15) / 16 * 16;
   plan.T = p.n_ctx + p.R;
   plan.tiles_per_item = ceil_div(plan.T, kTile);
@@ -1205,6 +1205,8 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
     case 64: launch_tc<64>(mk, mv, a, s); break;
     case 80: launch_tc<80>(mk, mv, a, s); break;
     case 96: launch_tc<96>(mk, mv, a, s); break;
+    case 112: launch_tc<112>(mk, mv, a, s); break;
+    case 128: launch_tc<128>(mk, mv, a, s); break;
     default: return PVLM_ERR_UNSUPPORTED;
   }
   if (p.prof_event_end) cudaEventRecord((cudaEvent_t)p.prof_event_end, s);

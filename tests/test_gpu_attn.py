@@ -168,6 +168,15 @@ def test_mma_sync_path_still_matches(monkeypatch):
         run_case(qb, kb, vb, n_ctx)
 
 
+@pytest.mark.parametrize("Hq,Hkv,R", [(16, 2, 13), (16, 2, 16), (14, 2, 15)])
+def test_wide_row_groups_on_the_tensor_core_path(Hq, Hkv, R, monkeypatch):
+    """97..128 query rows per KV head (3 ring slots, 2 score buffers): long tile runs with several segments per CTA."""
+    monkeypatch.setenv("PVLM_TC_CTAS", "3")
+    n_ctx = 2100
+    qb, kb, vb = wl.make_qkv(Hq, Hkv, 128, R, n_ctx + R, sink=True, seed=500 + R)
+    run_case(qb, kb, vb, n_ctx)
+
+
 def test_head_dim_64_on_the_tensor_core_path(monkeypatch):
     """D = 64 runs the tcgen05 kernels on channels padded to 128 by the TMA's out-of-range fill: several layers,
     long tile runs on few CTAs (many segments per CTA), batched launch with mass rows."""
