@@ -579,7 +579,13 @@ def run_reference(args):
     cfg = wl.CONFIGS[args.config]
     attn_inputs = wl.attn_layer(cfg, cfg.cur_layer)
     acc_inputs = wl.accept_inputs(cfg)
-    n_heads = min(cfg.Hq, 4)
+    # The per-step sample is sized so that the whole run (K + W steps) ends within a few minutes: one calibration
+    # step on a single query head, then as many heads (1..4) as a budget of ~150 s over all steps allows.
+    t_cal = time.perf_counter()
+    oracle_sample_step(cfg, attn_inputs, acc_inputs, [0])
+    t_cal = time.perf_counter() - t_cal
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    n_heads = max(1, min(cfg.Hq, 4, int(budget / max(t_cal, 1e-3))))
     heads = list(range(n_heads))
     for _ in range(args.warmup):
         oracle_sample_step(cfg, attn_inputs, acc_inputs, heads)
