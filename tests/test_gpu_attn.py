@@ -67,6 +67,21 @@ def test_running_max_keeps_growing():
     run_case(wl.f32_to_bf16_bits(q), wl.f32_to_bf16_bits(k), wl.f32_to_bf16_bits(v), n_ctx)
 
 
+def test_extreme_score_ranges_stay_finite():
+    """Scores of magnitude ~1e3 (nearly one-hot rows) and a sudden jump of several hundred log2 units inside one
+    tile: the reference is replaced before anything is exponentiated, so nothing overflows."""
+    Hq, Hkv, D, n_ctx, R = 8, 2, 128, 1500, 5
+    T = n_ctx + R
+    rq, rk, rv = (np.random.Generator(np.random.Philox(key=[11, i])) for i in range(3))
+    q, k, v = wl.make_qkv_f32(Hq, Hkv, D, R, T, False, rq, rk, rv)
+    o, lse, mass = run_case(wl.f32_to_bf16_bits(8 * q), wl.f32_to_bf16_bits(8 * k), wl.f32_to_bf16_bits(v), n_ctx)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all() and torch.isfinite(mass).all()
+    k2 = k.copy()
+    k2[700:703, :, :] *= 60.0                     # three keys whose scores dwarf everything seen before
+    o, lse, mass = run_case(wl.f32_to_bf16_bits(q), wl.f32_to_bf16_bits(k2), wl.f32_to_bf16_bits(v), n_ctx)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all() and torch.isfinite(mass).all()
+
+
 def test_custom_scale_and_no_mass():
     qb, kb, vb = wl.make_qkv(8, 4, 64, 3, 203, sink=False, seed=21)
     run_case(qb, kb, vb, 200, scale=0.07)
