@@ -312,6 +312,7 @@ def run_ours(args):
         draft_report = draft_stream_leg(cfg, dev, torch, binding, wl, Q, K, V, O, lse, mass, w, pp, pc, args)
         decode_report = decode_pipeline_leg(cfg, dev, torch, binding, Q, K, V, O, args)
         rate_report = acceptance_rate_leg(cfg, dev, torch, binding)
+        sim_report = similarity_leg(cfg, dev, torch, binding)
 
     total_ms, e2e_ms = max_over_ranks(dist, torch, [total_ms, e2e_ms], dev)
 
@@ -363,6 +364,7 @@ def run_ours(args):
         out["draft_stream"] = draft_report
         out["decode_pipeline"] = decode_report
         out["acceptance_rate"] = rate_report
+        out["similarity_criterion"] = sim_report
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, w)
     print(json.dumps(out))
@@ -429,6 +431,30 @@ def draft_stream_leg(cfg, dev, torch, binding, wl, Q, K, V, O, lse, mass, w, pp,
             "verify_step_us_alone": v_alone, "draft_window_us_alone": d_alone,
             "verify_step_us_concurrent": v_con, "draft_window_us_concurrent": d_con,
             "both_us_concurrent": max(v_con, d_con), "both_us_serial": v_alone + d_alone}
+
+
+def similarity_leg(cfg, dev, torch, binding):
+    """The paper's own UV-Prune signal (Eq. 1-2) on one early layer's token representations of this config's shape:
+    sum_j cos(V_i, X_j) for the m visual rows against the n text rows, (m + 2n) * d_model * 2 bytes per call; the
+    variation score needs two such calls (first and last early layer) before the same select / gather."""
+    m, n, d = cfg.m, cfg.n_text, cfg.d_model
+    g = torch.Generator(device=dev)
+    g.manual_seed(9)
+    hs = [torch.randn((m + n, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16) for _ in range(4)]
+    sim = torch.empty(m, device=dev)
+    for i in range(4):
+        binding.uvprune_similarity(hs[i], 0, m, m, n, out=sim)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 20
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(reps):
+        binding.uvprune_similarity(hs[i % 4], 0, m, m, n, out=sim)      # four buffers (1.4 GB) rotate: no L2 reuse
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    byts = (m + 2 * n) * d * 2
+    return {"visual_rows": m, "text_rows": n, "d_model": d, "us": ms * 1e3, "bytes": byts, "gbs": byts / ms / 1e6}
 
 
 def acceptance_rate_leg(cfg, dev, torch, binding, n_tok=1024):
