@@ -8,7 +8,6 @@ namespace pvlm {
 
 namespace {
 
-constexpr int kSimRowChunks = 64;      // text rows are summed in this many independent slices
 
 struct SimArgs {
   const __nv_bfloat16* h;
@@ -16,7 +15,7 @@ struct SimArgs {
   int vis_start, m, text_start, n, d;
   float* sim;
   float* inv_norm;   // [n]
-  float* u_part;     // [kSimRowChunks][d]
+  float* u_part;     // [text CTAs][d]
   float* u;          // [d]
 };
 
@@ -36,49 +35,93 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// 1 / |X_j| per text row (0 for a zero row): one warp per row.
-__global__ void __launch_bounds__(256) sim_text_norm_kernel(const SimArgs a) {
-  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (row >= a.n) return;
-  const uint4* src = reinterpret_cast<const uint4*>(a.h + (long long)(a.text_start + row) * a.row_stride);
-  float acc = 0.f;
-  for (int c = lane; c < a.d / 8; c += 32) {
-    float f[8];
-    unpack8(__ldg(src + c), f);
+constexpr int kSimRowsPerCta = 8;      // text rows per CTA of the text pass (one per warp)
+
+// Text pass, one read of the text rows from HBM: a CTA takes 8 consecutive rows; each warp computes 1 / |X_j| of
+// one of them (0 for a zero row), then every thread sums its 8-channel groups over the 8 rows in row order
+// (the rows come back from L1 / L2) and writes one partial of u.  Fixed order everywhere: deterministic.
+__global__ void __launch_bounds__(256) sim_text_kernel(const SimArgs a) {
+  __shared__ float s_inv[kSimRowsPerCta];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int r0 = blockIdx.x * kSimRowsPerCta;
+  for (int k = warp; k < kSimRowsPerCta; k += 8) {
+    const int row = r0 + k;
+    float acc = 0.f;
+    if (row < a.n) {
+      const uint4* src = reinterpret_cast<const uint4*>(a.h + (long long)(a.text_start + row) * a.row_stride);
+      const int n4 = a.d / 8;
+      int c = lane;
+      for (; c + 7 * 32 < n4; c += 8 * 32) {              // eight 16-byte loads in flight per lane
+        uint4 v[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+        for (int i = 0; i < 8; ++i) v[i] = __ldg(src + c + i * 32);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float f[8];
+          unpack8(v[i], f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+        }
+      }
+      for (; c < n4; c += 32) {
+        float f[8];
+        unpack8(__ldg(src + c), f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+      }
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) s_inv[k] = acc > 0.f ? rsqrtf(acc) : 0.f;
   }
-  acc = warp_sum(acc);
-  if (lane == 0) a.inv_norm[row] = acc > 0.f ? rsqrtf(acc) : 0.f;
+  __syncthreads();
+  const int rows = min(kSimRowsPerCta, a.n - r0);
+  for (int c = threadIdx.x; c < a.d / 8; c += 256) {
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    uint4 v[kSimRowsPerCta];
+#pragma unroll
+    for (int k = 0; k < kSimRowsPerCta; ++k)                 // all eight loads in flight, then a fixed-order sum
+      v[k] = k < rows ? __ldg(reinterpret_cast<const uint4*>(a.h + (long long)(a.text_start + r0 + k) * a.row_stride) + c)
+                      : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int k = 0; k < kSimRowsPerCta; ++k) {
+      const float w = k < rows ? s_inv[k] : 0.f;
+      float f[8];
+      unpack8(v[k], f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = fmaf(f[e], w, acc[e]);
+    }
+    float* dst = a.u_part + (long long)blockIdx.x * a.d + c * 8;
+    *reinterpret_cast<float4*>(dst) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+  }
 }
 
-// Partial column sums of the normalised text rows: grid (ceil(d/8/256), kSimRowChunks).
-__global__ void __launch_bounds__(256) sim_text_sum_kernel(const SimArgs a) {
-  const int c = blockIdx.x * 256 + threadIdx.x;       // 8-channel group
-  if (c >= a.d / 8) return;
-  const int rows_per = (a.n + kSimRowChunks - 1) / kSimRowChunks;
-  const int r0 = blockIdx.y * rows_per, r1 = min(a.n, r0 + rows_per);
-  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll 8
-  for (int r = r0; r < r1; ++r) {
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(a.h + (long long)(a.text_start + r) * a.row_stride) + c);
-    const float w = a.inv_norm[r];
-    float f[8];
-    unpack8(v, f);
+// u = sum of the partials: a CTA owns 32 channels (a lane each); its 8 warps take the partials round-robin with eight
+// loads in flight each, and their sums are merged in warp order.  The order is fixed: deterministic.
+__global__ void __launch_bounds__(256) sim_text_reduce_kernel(const SimArgs a, int n_part) {
+  __shared__ float s_sum[8][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + lane;
+  float sacc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (c < a.d) {
+    int k = warp;
+    for (; k + 56 < n_part; k += 64) {                     // eight loads in flight per lane
+      float v[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = fmaf(f[e], w, acc[e]);
+      for (int i = 0; i < 8; ++i) v[i] = a.u_part[(long long)(k + 8 * i) * a.d + c];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sacc[i] += v[i];
+    }
+    for (; k < n_part; k += 8) sacc[0] += a.u_part[(long long)k * a.d + c];
   }
-  float* dst = a.u_part + (long long)blockIdx.y * a.d + c * 8;
+  s_sum[warp][lane] = ((sacc[0] + sacc[1]) + (sacc[2] + sacc[3])) + ((sacc[4] + sacc[5]) + (sacc[6] + sacc[7]));
+  __syncthreads();
+  if (warp == 0 && c < a.d) {
+    float t = s_sum[0][lane];
 #pragma unroll
-  for (int e = 0; e < 8; ++e) dst[e] = acc[e];
-}
-
-__global__ void __launch_bounds__(256) sim_text_reduce_kernel(const SimArgs a) {
-  const int c = blockIdx.x * 256 + threadIdx.x;
-  if (c >= a.d) return;
-  float acc = 0.f;
-  for (int k = 0; k < kSimRowChunks; ++k) acc += a.u_part[(long long)k * a.d + c];
-  a.u[c] = acc;
+    for (int w = 1; w < 8; ++w) t += s_sum[w][lane];
+    a.u[c] = t;
+  }
 }
 
 // sim_i = (V_i . u) / |V_i|: u staged in shared memory, one warp per visual row, 16-byte loads.
@@ -90,16 +133,25 @@ __global__ void __launch_bounds__(256) sim_visual_kernel(const SimArgs a) {
   for (int row = blockIdx.x * 8 + warp; row < a.m; row += gridDim.x * 8) {
     const uint4* src = reinterpret_cast<const uint4*>(a.h + (long long)(a.vis_start + row) * a.row_stride);
     float dot = 0.f, nrm = 0.f;
-#pragma unroll 4
-    for (int c = lane; c < a.d / 8; c += 32) {
+    auto take = [&](const uint4& v, int c) {
       float f[8];
-      unpack8(__ldg(src + c), f);
+      unpack8(v, f);
       const float4 u0 = *reinterpret_cast<const float4*>(s_u + c * 8), u1 = *reinterpret_cast<const float4*>(s_u + c * 8 + 4);
       dot = fmaf(f[0], u0.x, dot); dot = fmaf(f[1], u0.y, dot); dot = fmaf(f[2], u0.z, dot); dot = fmaf(f[3], u0.w, dot);
       dot = fmaf(f[4], u1.x, dot); dot = fmaf(f[5], u1.y, dot); dot = fmaf(f[6], u1.z, dot); dot = fmaf(f[7], u1.w, dot);
 #pragma unroll
       for (int e = 0; e < 8; ++e) nrm = fmaf(f[e], f[e], nrm);
+    };
+    const int n4 = a.d / 8;
+    int c = lane;
+    for (; c + 9 * 32 < n4; c += 10 * 32) {                 // ten 16-byte loads in flight per lane
+      uint4 v[10];
+#pragma unroll
+      for (int i = 0; i < 10; ++i) v[i] = __ldg(src + c + i * 32);
+#pragma unroll
+      for (int i = 0; i < 10; ++i) take(v[i], c + i * 32);
     }
+    for (; c < n4; c += 32) take(__ldg(src + c), c);
     dot = warp_sum(dot);
     nrm = warp_sum(nrm);
     if (lane == 0) a.sim[row] = nrm > 0.f ? dot * rsqrtf(nrm) : 0.f;
@@ -108,9 +160,10 @@ __global__ void __launch_bounds__(256) sim_visual_kernel(const SimArgs a) {
 
 }  // namespace
 
+static int sim_text_parts(int n) { return n > 0 ? ceil_div(n, kSimRowsPerCta) : 1; }
+
 size_t similarity_workspace(const pvlm_similarity_params& p) {
-  return align_up((size_t)(p.n > 0 ? p.n : 1) * 4, 256) + align_up((size_t)kSimRowChunks * p.d * 4, 256) +
-         align_up((size_t)p.d * 4, 256);
+  return align_up((size_t)sim_text_parts(p.n) * p.d * 4, 256) + align_up((size_t)p.d * 4, 256);
 }
 
 pvlm_status launch_similarity(const pvlm_similarity_params& p, cudaStream_t s) {
@@ -120,12 +173,12 @@ pvlm_status launch_similarity(const pvlm_similarity_params& p, cudaStream_t s) {
   a.vis_start = p.vis_start; a.m = p.m; a.text_start = p.text_start; a.n = p.n; a.d = p.d;
   a.sim = p.sim;
   char* ws = (char*)p.workspace;
-  a.inv_norm = (float*)ws;
-  a.u_part = (float*)(ws + align_up((size_t)(p.n > 0 ? p.n : 1) * 4, 256));
-  a.u = (float*)((char*)a.u_part + align_up((size_t)kSimRowChunks * p.d * 4, 256));
-  if (p.n > 0) sim_text_norm_kernel<<<ceil_div(p.n, 8), 256, 0, s>>>(a);
-  sim_text_sum_kernel<<<dim3(ceil_div(p.d / 8, 256), kSimRowChunks), 256, 0, s>>>(a);
-  sim_text_reduce_kernel<<<ceil_div(p.d, 256), 256, 0, s>>>(a);
+  const int parts = sim_text_parts(p.n);
+  a.u_part = (float*)ws;
+  a.u = (float*)(ws + align_up((size_t)parts * p.d * 4, 256));
+  a.inv_norm = nullptr;
+  if (p.n > 0) sim_text_kernel<<<parts, 256, 0, s>>>(a);
+  sim_text_reduce_kernel<<<ceil_div(p.d, 32), 256, 0, s>>>(a, p.n > 0 ? parts : 0);
   if (p.m > 0) {
     int blocks = ceil_div(p.m, 8);
     if (blocks > kNumSMs * 16) blocks = kNumSMs * 16;
