@@ -366,7 +366,11 @@ def run_ours(args):
         out["acceptance_rate"] = rate_report
         out["similarity_criterion"] = sim_report
     if world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(cfg, w)
+        torch.cuda.synchronize()
+        li = cfg.cur_layer if L > 1 else 0                      # the layer whose K/V are host-generated and oracle-checkable
+        gpu = {"o": O[li].float().cpu().numpy(), "mass": mass_cur.cpu().numpy(), "lse": lse[li].cpu().numpy(),
+               "n_accept": int(outs["n_accept"].item()), "out_tokens": outs["out_tokens"].cpu().numpy().ravel()}
+        out["cpu_baseline"] = cpu_baseline(cfg, w, gpu if (args.layers == 0 or li < L) else None)
     print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
@@ -571,14 +575,16 @@ def oracle_sample_step(cfg, attn_inputs, acc_inputs, heads):
     from oracle.accept import spec_accept as o_accept
     q, k, v = attn_inputs
     t0 = time.perf_counter()
-    _, _, mass = o_attn(q, k, v, cfg.n_ctx, heads=heads)
+    o_ref, lse_ref, mass = o_attn(q, k, v, cfg.n_ctx, heads=heads)
     t1 = time.perf_counter()
     idx = select_topk(score_fp32(mass.astype(np.float32), None, 0, cfg.m), cfg.k_keep)
     gather_rows(k[None], 0, cfg.m, idx)
     gather_rows(v[None], 0, cfg.m, idx)
     t2 = time.perf_counter()
-    o_accept(*acc_inputs)
+    acc = o_accept(*acc_inputs)
     t3 = time.perf_counter()
+    oracle_sample_step.last = {"o": o_ref, "lse": lse_ref, "mass": mass, "n_accept": int(acc["n_accept"]),
+                               "out_tokens": np.asarray(acc["out_tokens"])}
     return t1 - t0, t2 - t1, t3 - t2
 
 
@@ -596,22 +602,34 @@ def cpu_threads():
         return os.cpu_count() or 1
 
 
-def cpu_baseline(cfg, w=None):
+def cpu_baseline(cfg, w=None, gpu=None):
     """The oracle as it stands on a bounded sample: every query head of a few layers (about 10-30 s of CPU
-    work at the 32k config), one select+gather per sampled layer, the full accept; scaled to all layers."""
+    work at the 32k config), one select+gather per sampled layer, the full accept; scaled to all layers.
+    The first sampled layer is the one the bench's mass row and o come from, so the timed GPU results of that layer
+    (and the accept outcome) are compared with the oracle's here: `parity` in the returned object."""
     from paper_2603_19610_b200 import workloads as wl
     n_sample = min(cfg.n_layers, 4) if cfg.n_layers > 1 else 1
     acc_inputs = wl.accept_inputs(cfg)
     heads = list(range(cfg.Hq))
     ta = tp = tc = 0.0
+    parity = None
     for i in range(n_sample):
         layer = (cfg.cur_layer + i) % cfg.n_layers
         parts = oracle_sample_step(cfg, wl.attn_layer(cfg, layer), acc_inputs, heads)
         ta += parts[0]
         tp += parts[1]
         tc = parts[2]
+        if i == 0 and gpu is not None:
+            ref = oracle_sample_step.last
+            o_ratio = float((np.abs(gpu["o"] - ref["o"]) / (1e-2 + 2e-2 * np.abs(ref["o"]))).max())
+            mass_rel = float((np.abs(gpu["mass"] - ref["mass"]) / (np.abs(ref["mass"]) + 1e-300)).max())
+            lse_abs = float(np.abs(gpu["lse"] - ref["lse"]).max())
+            acc_ok = gpu["n_accept"] == ref["n_accept"] and bool((gpu["out_tokens"] == ref["out_tokens"]).all())
+            parity = {"layer": layer, "o_error_over_tolerance": o_ratio, "mass_max_rel_err": mass_rel, "lse_max_abs_err": lse_abs,
+                      "accept_matches": acc_ok,
+                      "ok": bool(o_ratio <= 1.0 and mass_rel <= 1e-4 and lse_abs <= 1e-4 and acc_ok)}
     est = (ta + tp) / n_sample * cfg.n_layers + tc
-    return {"value": est * 1e6, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+    return {"value": est * 1e6, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "parity": parity,
             "sample": f"oracle timed on all {cfg.Hq} query heads of {n_sample} layer(s) ({ta:.2f} s), their select+gather "
                       f"({tp:.3f} s) and the full accept ({tc:.3f} s); attention and gather scaled to {cfg.n_layers} layers"}
 
