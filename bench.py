@@ -344,8 +344,8 @@ def run_ours(args):
         "e2e": {"value": aggregate_us_per_step(e2e_ms, args.steps, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "KV cache of the committed context is resident device state; step inputs (Q, window K/V rows, "
                         "logits, drafts, uniforms) come from pinned host memory, results (O, kept indices, tokens) go back"},
-        # per step: attention main + merge + mass + mass reduce, select, gather (two launches in the fused step), 4 accept kernels
-        "gpu_launches": args.steps * (10 if args.serial_step else 11),
+        # per step: attention main + merge + mass + mass reduce, select, gather (two launches in the fused step), 2 accept kernels
+        "gpu_launches": args.steps * (8 if args.serial_step else 9),
         "stages_note": "stage times come from a separate pass that runs the stages as three serial calls; the timed step is one "
                        "call in which the accept stage and the selection-independent part of the gather run on a second stream",
         "stages_us": {"attention": attn_avg_ms * 1e3, "prune_select_gather": sum(prune_ms) / len(prune_ms) * 1e3,

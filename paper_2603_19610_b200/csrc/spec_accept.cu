@@ -4,6 +4,9 @@
 //   accept_scan : merge chunks -> lse per row; p(x_t), q(x_t); first rejection n
 //   resid_sums  : row pair n only: per-chunk sums of max(0, p-q) and of p (fp64)
 //   resid_pick  : inverse CDF over the chunk sums, then inside the crossing chunk
+// Two launches: the CTA of row_stats / resid_sums that finishes last for a sequence (a ticket counter in the
+// workspace) goes straight on to that sequence's accept_scan / resid_pick, so the two small single-CTA
+// steps cost no launch of their own.
 #include "pvlm_common.cuh"
 
 namespace pvlm {
@@ -30,6 +33,7 @@ struct AccArgs {
   double* lse;        // [batch][rows]
   double* csum;       // [batch][n_samp_chunks][2]
   int* clast;         // [batch][n_samp_chunks][2]
+  int* tickets;       // [batch][2] CTAs finished per sequence in the two launches (zeroed per call, reset by the last CTA)
   int n_stat_chunks, n_samp_chunks;
 };
 
@@ -51,6 +55,9 @@ __device__ __forceinline__ void merge_ml(float& m, float& l, float m2, float l2,
   l = l * ex2f((m - mn) * c) + l2 * ex2f((m2 - mn) * c);
   m = mn;
 }
+
+__device__ void accept_scan_body(const AccArgs& a, int b);
+__device__ void resid_pick_body(const AccArgs& a, int b);
 
 __global__ void __launch_bounds__(kStatThreads) row_stats_kernel(const AccArgs a) {
   const int chunk = blockIdx.x, row = blockIdx.y, b = blockIdx.z;
@@ -85,14 +92,23 @@ __global__ void __launch_bounds__(kStatThreads) row_stats_kernel(const AccArgs a
   __shared__ float sm[kStatThreads / 32], sl[kStatThreads / 32];
   if ((threadIdx.x & 31) == 0) { sm[threadIdx.x >> 5] = m; sl[threadIdx.x >> 5] = l; }
   __syncthreads();
+  __shared__ int s_is_last;
   if (threadIdx.x == 0) {
     for (int w = 1; w < kStatThreads / 32; ++w) merge_ml(m, l, sm[w], sl[w], c);
     a.stats[((long long)b * a.rows + row) * a.n_stat_chunks + chunk] = make_float2(m, l);
+    __threadfence();                                   // the partial is visible before the ticket is taken
+    const int ticket = atomicAdd(&a.tickets[2 * b], 1);
+    s_is_last = ticket == a.rows * a.n_stat_chunks - 1;
+    if (s_is_last) a.tickets[2 * b] = 0;
+  }
+  __syncthreads();
+  if (s_is_last) {                                     // every partial of this sequence has been written
+    __threadfence();
+    accept_scan_body(a, b);
   }
 }
 
-__global__ void __launch_bounds__(1024) accept_scan_kernel(const AccArgs a) {
-  const int b = blockIdx.x;
+__device__ void accept_scan_body(const AccArgs& a, const int b) {
   const float c = a.inv_temp * kLog2e;
   __shared__ int s_reject[64];
   // one warp per logit row: lanes take chunk partials round-robin, then a fixed-order butterfly merge
@@ -101,7 +117,7 @@ __global__ void __launch_bounds__(1024) accept_scan_kernel(const AccArgs a) {
     const int lane = threadIdx.x & 31;
     float m = -INFINITY, l = 0.f;
     for (int ch = lane; ch < a.n_stat_chunks; ch += 32) {
-      const float2 v = st[ch];
+      const float2 v = __ldcg(st + ch);                // written by other CTAs: read through L2
       merge_ml(m, l, v.x, v.y, c);
     }
 #pragma unroll
@@ -199,10 +215,21 @@ __global__ void __launch_bounds__(kSampThreads) resid_sums_kernel(const AccArgs 
     a.csum[o] = sr; a.csum[o + 1] = sp;
     a.clast[o] = lr; a.clast[o + 1] = lp;
   }
+  __shared__ int s_is_last;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const int ticket = atomicAdd(&a.tickets[2 * b + 1], 1);
+    s_is_last = ticket == a.n_samp_chunks - 1;
+    if (s_is_last) a.tickets[2 * b + 1] = 0;
+  }
+  __syncthreads();
+  if (s_is_last) {
+    __threadfence();
+    resid_pick_body(a, b);
+  }
 }
 
-__global__ void __launch_bounds__(kSampThreads) resid_pick_kernel(const AccArgs a) {
-  const int b = blockIdx.x;
+__device__ void resid_pick_body(const AccArgs& a, const int b) {
   const int n = a.n_accept[b];
   __shared__ int s_chunk, s_fallback, s_pick;
   __shared__ double s_base, s_target;
@@ -225,10 +252,10 @@ __global__ void __launch_bounds__(kSampThreads) resid_pick_kernel(const AccArgs 
   double zr_part = 0.0, zp_part = 0.0;
   int last_r = -1, last_p = -1;
   for (int ch = threadIdx.x; ch < a.n_samp_chunks; ch += kSampThreads) {
-    zr_part += cs[2 * ch];
-    zp_part += cs[2 * ch + 1];
-    last_r = max(last_r, cl[2 * ch]);
-    last_p = max(last_p, cl[2 * ch + 1]);
+    zr_part += __ldcg(cs + 2 * ch);                    // written by other CTAs: read through L2
+    zp_part += __ldcg(cs + 2 * ch + 1);
+    last_r = max(last_r, __ldcg(cl + 2 * ch));
+    last_p = max(last_p, __ldcg(cl + 2 * ch + 1));
   }
   const double zr = block_sum(zr_part);
   const int mode = (zr > 0.0) ? 0 : 1;             // no residual weight at all => draw from p
@@ -240,7 +267,7 @@ __global__ void __launch_bounds__(kSampThreads) resid_pick_kernel(const AccArgs 
   double run_base = 0.0;
   for (int c0 = 0; c0 < a.n_samp_chunks; c0 += kSampThreads) {
     const int ch = c0 + threadIdx.x;
-    const double v = ch < a.n_samp_chunks ? cs[2 * ch + mode] : 0.0;
+    const double v = ch < a.n_samp_chunks ? __ldcg(cs + 2 * ch + mode) : 0.0;
     double incl = v;
 #pragma unroll
     for (int sh = 1; sh < 32; sh <<= 1) {
@@ -302,7 +329,7 @@ __global__ void __launch_bounds__(kSampThreads) resid_pick_kernel(const AccArgs 
   }
   if (mine != 0x7fffffff) atomicMin(&s_pick, mine);
   __syncthreads();
-  if (threadIdx.x == 0) *out = (s_pick != 0x7fffffff) ? s_pick : cl[2 * chunk + mode];
+  if (threadIdx.x == 0) *out = (s_pick != 0x7fffffff) ? s_pick : __ldcg(cl + 2 * chunk + mode);
 }
 
 __global__ void __launch_bounds__(256) write_probs_kernel(const AccArgs a) {
@@ -330,9 +357,9 @@ bool make_accept_plan(const pvlm_accept_params& p, AcceptPlan& plan) {
   size_t off = 0;
   plan.off_stats = off; off += align_up((size_t)p.batch * plan.rows * plan.n_stat_chunks * 8, 256);
   plan.off_lse = off;   off += align_up((size_t)p.batch * plan.rows * 8, 256);
-  plan.off_n = off;
   plan.off_csum = off;  off += align_up((size_t)p.batch * plan.n_samp_chunks * 2 * 8, 256);
   plan.off_clast = off; off += align_up((size_t)p.batch * plan.n_samp_chunks * 2 * 4, 256);
+  plan.off_n = off;     off += align_up((size_t)p.batch * 2 * 4, 256);       // ticket counters
   plan.total = off;
   return true;
 }
@@ -355,11 +382,12 @@ pvlm_status launch_spec_accept(const pvlm_accept_params& p, const AcceptPlan& pl
   a.lse = (double*)(ws + plan.off_lse);
   a.csum = (double*)(ws + plan.off_csum);
   a.clast = (int*)(ws + plan.off_clast);
+  a.tickets = (int*)(ws + plan.off_n);
   a.n_stat_chunks = plan.n_stat_chunks; a.n_samp_chunks = plan.n_samp_chunks;
-  row_stats_kernel<<<dim3(plan.n_stat_chunks, plan.rows, p.batch), kStatThreads, 0, s>>>(a);
-  accept_scan_kernel<<<p.batch, plan.rows > 32 ? 1024 : (plan.rows > 8 ? 512 : 128), 0, s>>>(a);
-  resid_sums_kernel<<<dim3(plan.n_samp_chunks, p.batch), kSampThreads, 0, s>>>(a);
-  resid_pick_kernel<<<p.batch, kSampThreads, 0, s>>>(a);
+  const cudaError_t e = cudaMemsetAsync(a.tickets, 0, (size_t)p.batch * 2 * 4, s);
+  if (e != cudaSuccess) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+  row_stats_kernel<<<dim3(plan.n_stat_chunks, plan.rows, p.batch), kStatThreads, 0, s>>>(a);      // + accept scan
+  resid_sums_kernel<<<dim3(plan.n_samp_chunks, p.batch), kSampThreads, 0, s>>>(a);                // + pick
   if (p.probs_p || p.probs_q)
     write_probs_kernel<<<dim3(ceil_div(p.V, 256), plan.rows, p.batch), 256, 0, s>>>(a);
   return check_launch();
