@@ -479,24 +479,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             : "memory");
         return out != 0;
       };
+      // Stages Q of one (layer, KV head) item in the K-major 128B-swizzled layout and tells the issuer.
+      auto stage_q = [&](int item) {
+        const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
+        const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * a.D;
+        const int cpr = a.D >> 3;                        // 16-byte pieces per query row: 16, or 8 when D = 64
+        for (int idx = st; idx < a.rows * cpr; idx += kSoftmaxThreads) {
+          const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
+          const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
+          const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
+          *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val;
+        }
+        fence_proxy_async();
+        mbar_arrive(bar(Q_READY));
+      };
+      stage_q((int)(f_begin / Tt));
       for (long long f = f_begin; f < f_end; ++seg) {
         const int item = (int)(f / Tt), tile0 = (int)(f - (long long)item * Tt);
         const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
         const int n = (int)(seg_end - f);
-        const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
-        // ---- stage Q of this (layer, KV head) in the K-major 128B-swizzled layout ----
-        {
-          const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * a.D;
-          const int cpr = a.D >> 3;                        // 16-byte pieces per query row: 16, or 8 when D = 64
-          for (int idx = st; idx < a.rows * cpr; idx += kSoftmaxThreads) {
-            const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
-            const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
-            const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
-            *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val;
-          }
-          fence_proxy_async();
-          mbar_arrive(bar(Q_READY));
-        }
         if (t < NRP) m_s[t] = kNegBig;
 #pragma unroll
         for (int i = 0; i < NRP; ++i) l_loc[i] = 0.f;
@@ -658,6 +659,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         // both groups leave together: the exit vote is per group, so agree across groups here
         if (softmax_bar_or(aborted)) break;
+        // Both groups have read the scores of their last tiles, so every score MMA of this segment is done and Q is
+        // free: the next item's Q goes in now, and the issuer starts that segment's score MMAs while the epilogue
+        // below drains this segment's accumulators.
+        if (seg_end < f_end) stage_q(item + 1);
         // ---- segment epilogue: this group's partial O (fp32), and (m, l) per row ----
         ok &= mbar_wait(bar(O_FULL), seg & 1, s_abort);
         tc_fence_after();
