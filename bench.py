@@ -94,7 +94,7 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------
 # workload construction
 # --------------------------------------------------------------------------------------
-def build_workload(cfg, dev, torch):
+def build_workload(cfg, dev, torch, layout="token"):
     """Device-resident state and step inputs for one config.
 
     K/V content of the layers that feed the variation score (reference and current layer) is
@@ -104,8 +104,13 @@ def build_workload(cfg, dev, torch):
     L, T, Hkv, Hq, D, R = cfg.n_layers, cfg.T, cfg.Hkv, cfg.Hq, cfg.D, cfg.R
     g = torch.Generator(device=dev)
     g.manual_seed(wl.BASE_SEED + 100 * cfg.cid)
-    K = torch.empty((L, T, Hkv, D), dtype=torch.bfloat16, device=dev)
-    V = torch.empty_like(K)
+    if layout == "head":                  # [layer][kv_head][token][D] storage, handed on as a [layer][token][kv_head][D] view
+        K_base = torch.empty((L, Hkv, T, D), dtype=torch.bfloat16, device=dev)
+        V_base = torch.empty_like(K_base)
+        K, V = K_base.permute(0, 2, 1, 3), V_base.permute(0, 2, 1, 3)
+    else:
+        K_base = K = torch.empty((L, T, Hkv, D), dtype=torch.bfloat16, device=dev)
+        V_base = V = torch.empty_like(K)
     Q = torch.empty((L, R, Hq, D), dtype=torch.bfloat16, device=dev)
     bias = torch.from_numpy(wl.position_bias(T, cfg.sink)).to(dev)
     for l in range(L):
@@ -125,7 +130,7 @@ def build_workload(cfg, dev, torch):
         K[l].copy_(torch.from_numpy(k.view(np.int16)).view(torch.bfloat16))
         V[l].copy_(torch.from_numpy(v.view(np.int16)).view(torch.bfloat16))
     tl, dl, tok, u = wl.accept_inputs(cfg)
-    return dict(K=K, V=V, Q=Q, mass_layers=mass_layers, tl=tl, dl=dl, tok=tok, u=u)
+    return dict(K=K, V=V, K_base=K_base, V_base=V_base, Q=Q, mass_layers=mass_layers, tl=tl, dl=dl, tok=tok, u=u)
 
 
 def algorithmic_bytes(cfg):
@@ -174,7 +179,7 @@ def run_ours(args):
         import dataclasses
         cfg = dataclasses.replace(cfg, n_layers=args.layers, name=cfg.name + f"-truncated-to-{args.layers}L",
                                   cur_layer=min(cfg.cur_layer, args.layers - 1))
-    w = build_workload(cfg, dev, torch)
+    w = build_workload(cfg, dev, torch, args.kv_layout)
     L, T, R = cfg.n_layers, cfg.T, cfg.R
     K, V, Q = w["K"], w["V"], w["Q"]
     O = torch.empty_like(Q)
@@ -190,7 +195,13 @@ def run_ours(args):
         mass_ref, mass_cur = mass[0], mass[1]
     kept = torch.empty(cfg.k_keep, dtype=torch.int32, device=dev)
     S2 = T - cfg.m + cfg.k_keep
-    dK = torch.empty((L, S2, cfg.Hkv, cfg.D), dtype=torch.bfloat16, device=dev)
+    head_major = args.kv_layout == "head"
+    if head_major:                         # the gather then sees L * Hkv "layers" of 256-byte rows
+        src_k, src_v = w["K_base"].view(L * cfg.Hkv, T, 1, cfg.D), w["V_base"].view(L * cfg.Hkv, T, 1, cfg.D)
+        dK = torch.empty((L * cfg.Hkv, S2, 1, cfg.D), dtype=torch.bfloat16, device=dev)
+    else:
+        src_k, src_v = K, V
+        dK = torch.empty((L, S2, cfg.Hkv, cfg.D), dtype=torch.bfloat16, device=dev)
     dV = torch.empty_like(dK)
     tl = torch.from_numpy(w["tl"]).to(dev)
     dl = torch.from_numpy(w["dl"]).to(dev)
@@ -209,12 +220,13 @@ def run_ours(args):
     torch.cuda.synchronize()
     pa.prof_event_begin, pa.prof_event_end = k_ev[0].cuda_event, k_ev[1].cuda_event
     main_kernel_ms = []
-    pp = binding.prune_params(mass_cur, mass_ref, 0, cfg.m, cfg.k_keep, kept, None, K, V, dK, dV)
+    pp = binding.prune_params(mass_cur, mass_ref, 0, cfg.m, cfg.k_keep, kept, None, src_k, src_v, dK, dV)
     pc = binding.accept_params(tl, dl, tok, u, 1.0, outs)
 
     # host-side step inputs / outputs for the end-to-end leg (pinned)
-    pin = lambda t: t.cpu().pin_memory()
-    h_in = dict(h_q=pin(Q), h_k_window=pin(K[:, cfg.n_ctx:]), h_v_window=pin(V[:, cfg.n_ctx:]),
+    pin = lambda t: t.contiguous().cpu().pin_memory()
+    win = (lambda base: base[:, :, cfg.n_ctx:]) if head_major else (lambda base: base[:, cfg.n_ctx:])   # the window's own rows
+    h_in = dict(h_q=pin(Q), h_k_window=pin(win(w["K_base"])), h_v_window=pin(win(w["V_base"])),
                 h_target_logits=pin(tl), h_draft_logits=pin(dl), h_draft_tokens=pin(tok), h_uniforms=pin(u))
     h_out = dict(h_o=torch.empty(O.shape, dtype=O.dtype).pin_memory(),
                  h_n_accept=torch.empty(1, dtype=torch.int32).pin_memory(),
@@ -328,9 +340,9 @@ def run_ours(args):
     ab_kernel = L * (2 * T * cfg.Hkv * cfg.D * 2 + R * cfg.Hq * cfg.D * 2)      # K and V once, Q once; partials excluded
     achieved = ab_kernel / (kern_ms * 1e-3) / 1e9
     # DRAM traffic of one launch of the dominant kernel, from the ncu capture of that kernel summarised under
-    # profiles/: 544.50 MB (read + write) for 4 layers of the config-2
+    # profiles/: 545.71 MB (read + write) for 4 layers of the config-2
     # geometry, which grows in proportion to the layers processed.
-    traffic = 544.50e6 / 4 * L if cfg.cid == 2 else None
+    traffic = 545.71e6 / 4 * L if cfg.cid == 2 else None
     out = {
         "metric": METRIC, "value": aggregate_us_per_step(total_ms, args.steps, world), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
@@ -339,6 +351,7 @@ def run_ours(args):
         "config": {"workload": f"config{cfg.cid}:{cfg.name}", "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
                    "n_ctx": cfg.n_ctx, "gamma": cfg.gamma, "layers": L, "vocab": cfg.V, "keep": cfg.k_keep,
                    "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "kv_layout": "[layer][kv_head][token][D]" if head_major else "[layer][token][kv_head][D]",
                    "l2": f"per-step inputs {(ab_attn + ab_prune + ab_acc) / 1e9:.2f} GB >> 126 MB L2 (no flush needed)"},
         "clocks": clocks,
         "e2e": {"value": aggregate_us_per_step(e2e_ms, args.steps, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -681,6 +694,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-draft-stream", action="store_true", help="skip the draft-stream concurrency leg")
     ap.add_argument("--draft-sms", type=int, default=44, help="SMs left to the draft stream in the concurrency leg")
+    ap.add_argument("--kv-layout", choices=["token", "head"], default="head",
+                    help="KV cache storage: [layer][token][kv_head][D] or [layer][kv_head][token][D] (both through the ABI's strides)")
     ap.add_argument("--serial-step", action="store_true", help="time the step as three serial calls on one stream "
                     "(default: one call, accept stage on a second stream)")
     ap.add_argument("--decode-draft-sms", type=int, default=44, help="SMs of the draft stream in the decode-pipeline leg")

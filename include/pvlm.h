@@ -241,8 +241,11 @@ pvlm_status pvlm_spec_accept(const pvlm_accept_params *p, void *stream);
  * is 0 is skipped.  Every h_* pointer is a HOST pointer (pinned memory makes
  * the copies asynchronous) and may be NULL, which skips that copy:
  *   h_q            bf16 [n_layers][R][Hq][D]        -> attn.q
- *   h_k_window/v   bf16 [n_layers][R][Hkv][D]       -> attn.k / attn.v rows n_ctx.. (needs
- *                                                      kv_head_stride == D, kv_token_stride == Hkv*D)
+ *   h_k_window/v   bf16 [n_layers][R][Hkv][D]       -> attn.k / attn.v rows n_ctx.. of a token-major cache
+ *                                                      (kv_head_stride == D, kv_token_stride == Hkv*D), or
+ *                  bf16 [n_layers][Hkv][R][D]       -> the same rows of a head-major cache (kv_token_stride
+ *                                                      == D, kv_layer_stride == Hkv*kv_head_stride);
+ *                                                      other stride combinations: PVLM_ERR_UNSUPPORTED
  *   h_target_logits fp32 [batch][gamma+1][V] dense  -> accept.target_logits (dense strides required)
  *   h_draft_logits  fp32 [batch][gamma][V] dense    -> accept.draft_logits
  *   h_draft_tokens, h_uniforms                      -> accept.draft_tokens, accept.uniforms

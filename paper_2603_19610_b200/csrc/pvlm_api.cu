@@ -212,15 +212,27 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
       e = cudaMemcpy2DAsync(const_cast<void*>(a.q), (size_t)a.q_layer_stride * 2, p->h_q, q_layer, q_layer, a.n_layers,
                             cudaMemcpyHostToDevice, s);
     if (p->h_k_window || p->h_v_window) {
-      if (a.kv_head_stride != a.D || a.kv_token_stride != (long long)a.Hkv * a.D) return PVLM_ERR_UNSUPPORTED;
-      const size_t w_layer = (size_t)a.R * a.Hkv * a.D * 2;
-      const size_t row0 = (size_t)a.n_ctx * a.kv_token_stride * 2;
-      const size_t pitch = a.n_layers > 1 ? (size_t)a.kv_layer_stride * 2 : w_layer;
+      const bool token_major = a.kv_head_stride == a.D && a.kv_token_stride == (long long)a.Hkv * a.D;
+      const bool head_major = a.kv_token_stride == a.D && a.kv_head_stride >= (long long)(a.n_ctx + a.R) * a.D &&
+                              (a.n_layers == 1 || a.kv_layer_stride == (long long)a.Hkv * a.kv_head_stride);
+      size_t width, pitch, row0 = (size_t)a.n_ctx * a.kv_token_stride * 2;
+      int height;
+      if (token_major) {                   // host [n_layers][R][Hkv][D]: one piece of R rows per layer
+        width = (size_t)a.R * a.Hkv * a.D * 2;
+        pitch = a.n_layers > 1 ? (size_t)a.kv_layer_stride * 2 : width;
+        height = a.n_layers;
+      } else if (head_major) {             // host [n_layers][Hkv][R][D]: one piece of R rows per (layer, KV head)
+        width = (size_t)a.R * a.D * 2;
+        pitch = (size_t)a.kv_head_stride * 2;
+        height = a.n_layers * a.Hkv;
+      } else {
+        return PVLM_ERR_UNSUPPORTED;
+      }
       if (p->h_k_window && ok())
-        e = cudaMemcpy2DAsync((char*)const_cast<void*>(a.k) + row0, pitch, p->h_k_window, w_layer, w_layer, a.n_layers,
+        e = cudaMemcpy2DAsync((char*)const_cast<void*>(a.k) + row0, pitch, p->h_k_window, width, width, height,
                               cudaMemcpyHostToDevice, s);
       if (p->h_v_window && ok())
-        e = cudaMemcpy2DAsync((char*)const_cast<void*>(a.v) + row0, pitch, p->h_v_window, w_layer, w_layer, a.n_layers,
+        e = cudaMemcpy2DAsync((char*)const_cast<void*>(a.v) + row0, pitch, p->h_v_window, width, width, height,
                               cudaMemcpyHostToDevice, s);
     }
   }

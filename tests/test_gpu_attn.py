@@ -128,7 +128,8 @@ def test_config1_full_size():
     run_case(q, k, v, cfg.n_ctx)
 
 
-def test_config2_full_size_batched_launch():
+@pytest.mark.parametrize("layout", ["head", "token"])
+def test_config2_full_size_batched_launch(layout):
     """Config-2 geometry at full context in the multi-layer launch configuration the bench
     times (4 of the 64 layers here; each layer checked in full against the oracle)."""
     cfg = wl.CONFIGS[2]
@@ -137,6 +138,10 @@ def test_config2_full_size_batched_launch():
     q = torch.stack([bf16_cuda(x[0]) for x in layers])
     k = torch.stack([bf16_cuda(x[1]) for x in layers])
     v = torch.stack([bf16_cuda(x[2]) for x in layers])
+    if layout == "head":                  # [layer][kv_head][token][D] storage (the bench's layout), passed through the strides
+        k = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        v = v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        assert k.stride(1) == cfg.D and k.stride(2) == cfg.T * cfg.D
     o, lse, mass = binding.verify_attn(q, k, v, cfg.n_ctx, want_mass=True)
     torch.cuda.synchronize()
     for l in range(L):

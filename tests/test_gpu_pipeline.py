@@ -145,6 +145,47 @@ def test_verify_step_host_buffers_config0():
     assert torch.equal(h_out["h_out_tokens"], acc_e["out_tokens"].cpu())
 
 
+def test_verify_step_host_buffers_head_major_cache():
+    """The step call with a head-major cache ([layer][kv_head][token][D]): the window's K/V rows arrive from a host
+    buffer laid out [layer][kv_head][R][D], the gather sees layer * kv_head pseudo-layers of D-element rows; results
+    equal those of the token-major calls."""
+    dev = torch.device("cuda", 0)
+    L, R, Hq, Hkv, D, n_ctx, m, k_keep = 3, 5, 8, 2, 128, 700, 600, 150
+    T = n_ctx + R
+    g = torch.Generator(device=dev); g.manual_seed(8)
+    mk = lambda *sh: torch.randn(sh, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    q, k, v = mk(L, R, Hq, D), mk(L, T, Hkv, D), mk(L, T, Hkv, D)
+    o_e, lse_e, mass_e = binding.verify_attn(q, k, v, n_ctx, want_mass=True, mass_layers=[0, 2])
+    kept_e, _, dk_e, dv_e = binding.uvprune_select_gather(mass_e[1], mass_e[0], 0, m, k_keep, k, v)
+    torch.cuda.synchronize()
+    kb = k.permute(0, 2, 1, 3).contiguous()                      # [L][Hkv][T][D]
+    vb = v.permute(0, 2, 1, 3).contiguous()
+    h_kw, h_vw = kb[:, :, n_ctx:].contiguous().cpu().pin_memory(), vb[:, :, n_ctx:].contiguous().cpu().pin_memory()
+    kb[:, :, n_ctx:] = 0; vb[:, :, n_ctx:] = 0
+    q2, o2 = torch.zeros_like(q), torch.zeros_like(q)
+    mass2 = torch.zeros_like(mass_e)
+    kept2 = torch.zeros(k_keep, dtype=torch.int32, device=dev)
+    S2 = T - m + k_keep
+    dk2 = torch.zeros((L * Hkv, S2, 1, D), dtype=torch.bfloat16, device=dev)
+    dv2 = torch.zeros_like(dk2)
+    pa = binding.attn_params(q2, kb.permute(0, 2, 1, 3), vb.permute(0, 2, 1, 3), n_ctx, o2, None, mass2, mass_layers=[0, 2])
+    pp = binding.prune_params(mass2[1], mass2[0], 0, m, k_keep, kept2, None, kb.view(L * Hkv, T, 1, D), vb.view(L * Hkv, T, 1, D), dk2, dv2)
+    h_in = dict(h_q=q.cpu().pin_memory(), h_k_window=h_kw, h_v_window=h_vw)
+    h_out = dict(h_o=torch.zeros(q.shape, dtype=torch.bfloat16).pin_memory(), h_kept_idx=torch.zeros(k_keep, dtype=torch.int32).pin_memory())
+    cs, ea, eb = torch.cuda.Stream(), torch.cuda.Event(), torch.cuda.Event()
+    ea.record(); eb.record()
+    torch.cuda.synchronize()
+    for overlap in (None, (cs, ea, eb)):
+        o2.zero_(); dk2.zero_(); dv2.zero_(); kept2.zero_(); kb[:, :, n_ctx:] = 0; vb[:, :, n_ctx:] = 0
+        binding.verify_step(pa, pp, None, host_in=h_in, host_out=h_out, device=dev, overlap=overlap)
+        torch.cuda.current_stream().synchronize()
+        assert torch.equal(kb.permute(0, 2, 1, 3), k) and torch.equal(vb.permute(0, 2, 1, 3), v)     # window rows landed
+        assert torch.equal(h_out["h_o"], o_e.cpu()) and torch.equal(h_out["h_kept_idx"], kept_e.cpu())
+        # compacted cache: [L * Hkv][S2][D] head-major against the token-major result [L][S2][Hkv][D]
+        assert torch.equal(dk2.view(L, Hkv, S2, D).permute(0, 2, 1, 3), dk_e)
+        assert torch.equal(dv2.view(L, Hkv, S2, D).permute(0, 2, 1, 3), dv_e)
+
+
 def test_verify_step_overlap_mode_splits_the_gather_correctly():
     """Overlap mode copies the rows outside the visual span on the second stream and the selected rows on the
     main stream: with rows before AND after the visual span the compacted caches must equal the one-call result."""
