@@ -398,8 +398,12 @@ def draft_stream_leg(cfg, dev, torch, binding, wl, Q, K, V, O, lse, mass, w, pp,
     S2 = cfg.T - cfg.m + cfg.k_keep
     g = torch.Generator(device=dev)
     g.manual_seed(7)
-    Kd = torch.randn((Ld, S2 + cfg.gamma, Hkv_d, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
-    Vd = torch.randn((Ld, S2 + cfg.gamma, Hkv_d, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    # the compacted draft cache, stored like the target's ([layer][kv_head][token][D] by default), seen as [layer][token][kv_head][D]
+    dshape = (Ld, Hkv_d, S2 + cfg.gamma, D) if args.kv_layout == "head" else (Ld, S2 + cfg.gamma, Hkv_d, D)
+    Kd = torch.randn(dshape, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    Vd = torch.randn(dshape, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    if args.kv_layout == "head":
+        Kd, Vd = Kd.permute(0, 2, 1, 3), Vd.permute(0, 2, 1, 3)
     Qd = torch.randn((Ld, 1, Hq_d, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
     Od = torch.empty_like(Qd)
     sD = torch.cuda.Stream(device=dev)
@@ -530,8 +534,11 @@ def decode_pipeline_leg(cfg, dev, torch, binding, Q, K, V, O, args):
     S2 = cfg.T - cfg.m + cfg.k_keep
     g = torch.Generator(device=dev)
     g.manual_seed(11)
-    Kd = torch.randn((Ld, S2 + gamma, Hkv_d, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
-    Vd = torch.randn((Ld, S2 + gamma, Hkv_d, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    dshape = (Ld, Hkv_d, S2 + gamma, D) if args.kv_layout == "head" else (Ld, S2 + gamma, Hkv_d, D)
+    Kd = torch.randn(dshape, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    Vd = torch.randn(dshape, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    if args.kv_layout == "head":
+        Kd, Vd = Kd.permute(0, 2, 1, 3), Vd.permute(0, 2, 1, 3)
     Qd = torch.randn((Ld, 1, Hq_d, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
     Od = torch.empty_like(Qd)
     P = n_tok + 2 * gamma + 1
@@ -572,7 +579,7 @@ def decode_pipeline_leg(cfg, dev, torch, binding, Q, K, V, O, args):
             "speedup_parallel_over_serial": t_ser / t_par,
             "note": "wall clock of the whole call (host round trips included); synthetic logit tables, so the acceptance "
                     "pattern is synthetic; same tokens in both orders. Both forwards are HBM-bound and share ONE GPU's "
-                    "HBM here, so overlapping them cannot beat running each on all SMs (the paper's gain comes from "
+                    "HBM here, so overlapping them gains little over running each on all SMs (the paper's gain comes from "
                     "draft and target sitting on different GPUs); the SM split is chosen so that both sides of a round "
                     "end together"}
 
