@@ -835,6 +835,108 @@ __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs 
   }
 }
 
+// The merge for items that many CTAs contributed to (short tile runs: few layers, long contexts).  Grid (items, rows):
+// a block per query row.  One thread per contributing CTA works out that CTA's slot; the row's (m, l) pairs go to
+// shared memory once, and the four warps take every fourth partial with four loads in flight.  Sums run in a fixed
+// order, so the result does not depend on timing.
+__global__ void __launch_bounds__(128) attn_tc_combine_many_kernel(const CombineArgs a) {
+  const int item = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __shared__ long long s_slot[2 * kNumSMs + 4];          // at most every CTA contributes two partials (-1: none)
+  __shared__ int s_n, s_c0;
+  __shared__ float s_m[4], s_l[4];
+  __shared__ float4 s_acc[4][32];
+  __shared__ float2 s_ml[2 * kNumSMs + 4];
+  {
+    // The CTAs whose tile ranges meet this item are consecutive: thread 0 finds the first and the last with a few
+    // divisions, then one thread per CTA works out that CTA's slot (-1: a CTA without tiles, possible when there
+    // are fewer tiles than CTAs).
+    const long long W = a.total_tiles, C = a.n_cta;
+    const long long lo = (long long)item * a.tiles_per_item, hi = lo + a.tiles_per_item;
+    auto bnd = [&](long long c) { return (W * c) / C; };
+    if (threadIdx.x == 0) {
+      long long c0 = (lo * C) / W;
+      while (c0 + 1 < C && bnd(c0 + 1) <= lo) ++c0;
+      while (c0 > 0 && bnd(c0) > lo) --c0;
+      long long c1 = ((hi - 1) * C) / W;
+      while (c1 + 1 < C && bnd(c1 + 1) < hi) ++c1;
+      while (c1 > c0 && bnd(c1) >= hi) --c1;
+      s_c0 = (int)c0;
+      s_n = 2 * (int)(c1 - c0 + 1);
+    }
+    __syncthreads();
+    const int cnt = s_n >> 1;
+    for (int k = threadIdx.x; k < cnt; k += 128) {
+      const long long c = s_c0 + k;
+      const long long b0 = bnd(c), b1 = bnd(c + 1);
+      const long long base = (b1 > b0 && b0 < hi && b1 > lo) ? (c * a.seg_max + (item - (int)(b0 / a.tiles_per_item))) * 2 : -1;
+      s_slot[2 * k] = base;
+      s_slot[2 * k + 1] = base < 0 ? -1 : base + 1;
+    }
+    __syncthreads();
+  }
+  const int n = s_n;
+  const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
+  auto store_row = [&](int row, float4 acc, float l, float mstar) {       // called by one warp
+    const float inv = 1.f / l;
+    const int r = row / a.G, g = row - r * a.G;
+    __nv_bfloat16* dst = a.o + (long long)layer * a.q_ls + ((long long)r * a.Hq + kvh * a.G + g) * a.D + lane * 4;
+    if (lane * 4 < a.D)
+      *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(acc.x * inv, acc.y * inv), pack2(acc.z * inv, acc.w * inv));
+    if (lane == 0) {
+      const long long li = (long long)layer * a.Hq * a.R + (kvh * a.G + g) * a.R + r;
+      const float v2 = mstar + log2f(l);
+      a.lse2[li] = v2;
+      if (a.lse) a.lse[li] = v2 * kLn2;
+    }
+  };
+  for (int row = blockIdx.y; row < a.rows; row += gridDim.y) {
+    // (m, l) of every partial of this row into shared memory; reference = largest m among those that saw a key
+    float mstar = -INFINITY;
+    for (int i = threadIdx.x; i < n; i += 128) {
+      const float2 ml = s_slot[i] >= 0 ? *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2)
+                                       : make_float2(kNegBig, 0.f);
+      s_ml[i] = ml;
+      if (ml.y > 0.f) mstar = fmaxf(mstar, ml.x);
+    }
+#pragma unroll
+    for (int sh = 16; sh >= 1; sh >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, sh));
+    if (lane == 0) s_m[warp] = mstar;
+    __syncthreads();
+    mstar = fmaxf(fmaxf(s_m[0], s_m[1]), fmaxf(s_m[2], s_m[3]));
+    float l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i0 = warp; i0 < n; i0 += 16) {               // a warp takes every fourth partial, four loads in flight
+      float4 o[4];
+      float w[4], lw[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + 4 * k;
+        const bool live = i < n && s_ml[i < n ? i : 0].y > 0.f;
+        w[k] = live ? ex2(s_ml[i].x - mstar) : 0.f;
+        lw[k] = live ? s_ml[i].y * w[k] : 0.f;
+        o[k] = live ? *reinterpret_cast<const float4*>(a.part_o + (s_slot[i] * a.nrp + row) * 128 + lane * 4)
+                    : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        l += lw[k];
+        acc.x += o[k].x * w[k]; acc.y += o[k].y * w[k]; acc.z += o[k].z * w[k]; acc.w += o[k].w * w[k];
+      }
+    }
+    s_acc[warp][lane] = acc;
+    if (lane == 0) s_l[warp] = l;
+    __syncthreads();
+    if (warp == 0) {
+      const float lt = ((s_l[0] + s_l[1]) + s_l[2]) + s_l[3];
+      float4 t = s_acc[0][lane];
+#pragma unroll
+      for (int w = 1; w < 4; ++w) { t.x += s_acc[w][lane].x; t.y += s_acc[w][lane].y; t.z += s_acc[w][lane].z; t.w += s_acc[w][lane].w; }
+      store_row(row, t, lt, mstar);
+    }
+    __syncthreads();
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Mass pass on the same machinery: S^T = K . Q^T only (no V, no P, no accumulator).  With the final
 // lse of every row known, a thread turns its key's scores into probabilities and adds them over the
@@ -1226,7 +1328,10 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
     const int items = p.Hkv * p.n_layers;
     int rows_y = 2048 / items;                            // enough blocks to fill the GPU, not tens of thousands
     rows_y = rows_y < 1 ? 1 : (rows_y > a.rows ? a.rows : rows_y);
-    attn_tc_combine_kernel<<<dim3(items, rows_y), 128, 0, s>>>(c);
+    // an item's tiles are spread over at most this many CTAs, each with two partials
+    const long long ctas_per_item = ((long long)plan.tiles_per_item * plan.n_cta + plan.total_tiles - 1) / plan.total_tiles + 1;
+    if (2 * ctas_per_item <= 8) attn_tc_combine_kernel<<<dim3(items, rows_y), 128, 0, s>>>(c);
+    else attn_tc_combine_many_kernel<<<dim3(items, rows_y), 128, 0, s>>>(c);
   }
   return check_launch();
 }
