@@ -213,7 +213,10 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
 // event trace of tiles 400..407 of CTA 0: status[64 + ev * 8 + (tile - 400)] = clock
 #define TRACE_T0(ev, j) { if (t == 0) TRACE(ev, j) }
 #define TRACE(ev, j) { if (blockIdx.x == 0 && (j) >= 400u && (j) < 408u) a.status[64 + (ev) * 8 + ((j) - 400u)] = (int)(clock64() & 0x7fffffff); }
+// phase marks of CTA 0 (first time each is reached): status[200 + i] = clock
+#define PHASE(i) { if (blockIdx.x == 0 && a.status[200 + (i)] == 0) a.status[200 + (i)] = (int)(clock64() & 0x7fffffff); }
 #else
+#define PHASE(i) {}
 #define PROF_DECL
 #define PROF_START
 #define PROF_ADD(i)
@@ -267,6 +270,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   auto bar = [&](int i) { return smem_addr(bars + i); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) PHASE(0)
 
   // ---- this CTA's range of the flattened tile sequence ----
   const long long W = a.total_tiles;
@@ -297,6 +301,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  if (tid == 0) PHASE(1)
   const uint32_t tmem_O = tmem;                    // O accumulators of the two softmax groups: columns [g*NRP, (g+1)*NRP)
   const uint32_t tmem_S = tmem + 2 * NRP;          // score buffers
 
@@ -494,6 +499,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         mbar_arrive(bar(Q_READY));
       };
       stage_q((int)(f_begin / Tt));
+      if (st == 0) PHASE(2)
       for (long long f = f_begin; f < f_end; ++seg) {
         const int item = (int)(f / Tt), tile0 = (int)(f - (long long)item * Tt);
         const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
@@ -516,6 +522,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           PROF_START
           ok &= mbar_wait(bar(S_FULL + sb), (j / NSB) & 1, s_abort);
           PROF_ADD(0)
+          if (st == 0) PHASE(3)
           TRACE_T0(4, j)
           tc_fence_after();
           // ---- scores of this key against all rows: x = s * scale - m (log2 domain), masked ----
@@ -654,10 +661,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           fence_proxy_async();
           tc_fence_before();                    // the score buffer has been read: this arrival also releases it
           mbar_arrive(bar(P_FULL + (j & 3)));
+          if (st == 0) PHASE(4)
           PROF_ADD(6)
           TRACE_T0(8, j)
         }
         // both groups leave together: the exit vote is per group, so agree across groups here
+        if (st == 0) PHASE(5)
         if (softmax_bar_or(aborted)) break;
         // Both groups have read the scores of their last tiles, so every score MMA of this segment is done and Q is
         // free: the next item's Q goes in now, and the issuer starts that segment's score MMAs while the epilogue
@@ -697,6 +706,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           a.part_ml[(slot * NRP + t) * 2 + 1] = has_tiles ? l : 0.f;
         }
         group_sync();
+        if (st == 0) PHASE(6)
         PROF_ADD(7)
         jt += n;
         f = seg_end;
@@ -709,6 +719,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // ---- teardown (every loop above is bounded, so every thread gets here) ----
   tc_fence_before();
   __syncthreads();
+  if (tid == 0) PHASE(7)
   if (*s_abort) {
     if (tid == 0) atomicExch(a.status, 1);
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);     // let copies / MMAs in flight land before TMEM is released
