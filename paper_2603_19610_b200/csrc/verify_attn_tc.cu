@@ -602,9 +602,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               for (int e = 0; e < 16; ++e) {
                 float v = __uint_as_float(raw[e]) * a.scale_log2;
                 if (e >= cw || (need_mask && rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16))) v = -INFINITY;
-#pragma unroll
-                for (int sh = 16; sh >= 1; sh >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, sh));
-                if (lane == 0 && e < cw) atomicMax(&newmax_s[c * 16 + e], f2ord(v));
+                // warp maximum in one instruction on the order-preserving integer image of the float
+                const int ov = __reduce_max_sync(0xffffffffu, f2ord(v));
+                if (lane == 0 && e < cw) atomicMax(&newmax_s[c * 16 + e], ov);
               }
             }
             group_sync();
