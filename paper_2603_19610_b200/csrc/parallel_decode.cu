@@ -24,7 +24,8 @@ struct DecodeLayout {
   size_t accept_ws, sample_ws, off_sample, off_small, total;
 };
 
-bool accept_block(const pvlm_decode_params& p, int gamma, int batch, pvlm_accept_params& c) {
+// Fills the fields of an accept call that are the same for every round: strides, sizes, temperature.
+void accept_block(const pvlm_decode_params& p, int gamma, int batch, pvlm_accept_params& c) {
   c = pvlm_accept_params{};
   c.target_row_stride = c.draft_row_stride = p.row_stride;
   c.target_batch_stride = c.draft_batch_stride = p.row_stride;
@@ -32,7 +33,6 @@ bool accept_block(const pvlm_decode_params& p, int gamma, int batch, pvlm_accept
   c.gamma = gamma;
   c.V = p.V;
   c.temperature = p.temperature;
-  return true;
 }
 
 bool make_layout(const pvlm_decode_params& p, DecodeLayout& l) {
