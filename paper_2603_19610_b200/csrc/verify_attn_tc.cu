@@ -325,6 +325,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const int item = (int)(f / Tt), tile = (int)(f - (long long)item * Tt);
           const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
           const uint32_t dst = smem_addr(sRing + slot * kTileBytes);
+          PHASE(8)
           mbar_expect_tx(full_bar, kTileBytes);
           tma_load_4d(dst, map, full_bar, 0, kvh, tile * kTile, layer);
           tma_load_4d(dst + kBoxBytes, map, full_bar, 64, kvh, tile * kTile, layer);
@@ -385,6 +386,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           ++u;
           PROF_START
           if (!wait_all(bar(K_FULL + (j & 3)), (j >> 2) & 1)) return false;
+          if (lane == 0) PHASE(10)
           PROF_ADD(0)
           TRACE(0, j)
           tc_fence_after();
@@ -400,6 +402,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             tc_commit(bar(EMPTY + slot));
           }
           __syncwarp();
+          if (lane == 0) PHASE(11)
           PROF_ADD(2)
           TRACE(1, j)
           return true;
@@ -409,6 +412,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
           const int n = (int)(seg_end - f);
           if (!wait_all(bar(Q_READY), seg & 1)) { ok = false; break; }
+          if (lane == 0) PHASE(9)
           tc_fence_after();
           int issued = 0;                                  // score tiles of this segment already issued
           for (int i = 0; i < n; ++i) {
@@ -489,11 +493,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
         const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * a.D;
         const int cpr = a.D >> 3;                        // 16-byte pieces per query row: 16, or 8 when D = 64
-        for (int idx = st; idx < a.rows * cpr; idx += kSoftmaxThreads) {
-          const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
-          const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
-          const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
-          *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val;
+        // every piece of a thread is loaded before the first is stored: one global round trip instead of up to eight
+        constexpr int QP = (NRP * 16 + kSoftmaxThreads - 1) / kSoftmaxThreads;
+        uint4 val[QP];
+#pragma unroll
+        for (int k = 0; k < QP; ++k) {
+          const int idx = st + k * kSoftmaxThreads;
+          if (idx < a.rows * cpr) {
+            const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
+            const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
+            val[k] = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < QP; ++k) {
+          const int idx = st + k * kSoftmaxThreads;
+          if (idx < a.rows * cpr) {
+            const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
+            *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val[k];
+          }
         }
         fence_proxy_async();
         mbar_arrive(bar(Q_READY));
