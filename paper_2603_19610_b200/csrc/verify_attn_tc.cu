@@ -213,16 +213,20 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
 // event trace of tiles 400..407 of CTA 0: status[64 + ev * 8 + (tile - 400)] = clock
 #define TRACE_T0(ev, j) { if (t == 0) TRACE(ev, j) }
 #define TRACE(ev, j) { if (blockIdx.x == 0 && (j) >= 400u && (j) < 408u) a.status[64 + (ev) * 8 + ((j) - 400u)] = (int)(clock64() & 0x7fffffff); }
-// phase marks of CTA 0 (first time each is reached): status[200 + i] = clock
-#define PHASE(i) { if (blockIdx.x == 0 && a.status[200 + (i)] == 0) a.status[200 + (i)] = (int)(clock64() & 0x7fffffff); }
 #else
-#define PHASE(i) {}
 #define PROF_DECL
 #define PROF_START
 #define PROF_ADD(i)
 #define PROF_DUMP(base) {}
 #define TRACE(ev, j)
 #define TRACE_T0(ev, j)
+#endif
+// phase marks of CTA 0 (first time each is reached): status[200 + i] = clock.  Also available without the per-tile
+// counters above (PVLM_TC_PHASES), which disturb a short run.
+#if defined(PVLM_TC_PROFILE) || defined(PVLM_TC_PHASES)
+#define PHASE(i) { if (blockIdx.x == 0 && a.status[200 + (i)] == 0) a.status[200 + (i)] = (int)(clock64() & 0x7fffffff); }
+#else
+#define PHASE(i) {}
 #endif
 
 // ---------------------------------------------------------------------------------------------
@@ -543,6 +547,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           if (st == 0) PHASE(3)
           TRACE_T0(4, j)
           tc_fence_after();
+          if (i == i_first) {
+            // First tile of this group's stream: instead of going through the reference-replacement path (row
+            // maxima over the tile, two group barriers), guess the reference from ONE key of the tile, its first:
+            // m = that key's score + 2 x threshold.  Any reference is valid; if another key of the tile beats the
+            // guess by more than the threshold (or the first key is masked for a row: then the "nothing seen"
+            // reference stays), the usual test below sends the group through the replacement path after all.
+            if (q4 == 0) {                             // the whole warp issues the (warp-collective) TMEM loads; lane 0 = the tile's first key
+#pragma unroll 1
+              for (int c = 0; c < NCH; ++c) {
+                uint32_t raw[16];
+                tmem_ld16(s_addr + c * 16, raw);
+                tmem_wait_ld();
+                reg_fence16(raw);
+                if (lane == 0) {
+#pragma unroll
+                  for (int e = 0; e < 16; ++e) {
+                    const bool masked = need_mask && rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16);
+                    if (!masked) m_s[c * 16 + e] = fmaf(__uint_as_float(raw[e]), a.scale_log2, 2.f * kRescaleThreshold);
+                  }
+                }
+                __syncwarp();
+              }
+            }
+            group_sync();
+          }
           // ---- scores of this key against all rows: x = s * scale - m (log2 domain), masked ----
           uint32_t xr[NCH][16];                       // TMEM loads land here and are converted in place
           float xmax;
