@@ -1126,11 +1126,24 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
         {
           const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * a.D;
           const int cpr = a.D >> 3;                        // 16-byte pieces per query row: 16, or 8 when D = 64
-          for (int idx = st; idx < a.rows * cpr; idx += kSoftmaxThreads) {
-            const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
-            const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
-            const uint4 val = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
-            *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val;
+          constexpr int QP = (NRP * 16 + kSoftmaxThreads - 1) / kSoftmaxThreads;
+          uint4 val[QP];                                   // all of a thread's pieces are in flight before the first store
+#pragma unroll
+          for (int k = 0; k < QP; ++k) {
+            const int idx = st + k * kSoftmaxThreads;
+            if (idx < a.rows * cpr) {
+              const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
+              const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
+              val[k] = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < QP; ++k) {
+            const int idx = st + k * kSoftmaxThreads;
+            if (idx < a.rows * cpr) {
+              const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
+              *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val[k];
+            }
           }
           if (st < 128) {
             float v = 1.0e30f;
