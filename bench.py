@@ -340,9 +340,9 @@ def run_ours(args):
     ab_kernel = L * (2 * T * cfg.Hkv * cfg.D * 2 + R * cfg.Hq * cfg.D * 2)      # K and V once, Q once; partials excluded
     achieved = ab_kernel / (kern_ms * 1e-3) / 1e9
     # DRAM traffic of one launch of the dominant kernel, from the ncu capture of that kernel summarised under
-    # profiles/: 545.71 MB (read + write) for 4 layers of the config-2
+    # profiles/: 544.04 MB (read + write) for 4 layers of the config-2
     # geometry, which grows in proportion to the layers processed.
-    traffic = 545.71e6 / 4 * L if cfg.cid == 2 else None
+    traffic = 544.04e6 / 4 * L if cfg.cid == 2 else None
     out = {
         "metric": METRIC, "value": aggregate_us_per_step(total_ms, args.steps, world), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
