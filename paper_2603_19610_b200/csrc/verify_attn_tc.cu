@@ -492,35 +492,40 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             : "memory");
         return out != 0;
       };
-      // Stages Q of one (layer, KV head) item in the K-major 128B-swizzled layout and tells the issuer.
-      auto stage_q = [&](int item) {
+      // Q of one (layer, KV head) item goes into the K-major 128B-swizzled layout in two steps, so that the global loads
+      // can be in flight while the thread does something else: q_load issues them, q_store writes shared memory and
+      // tells the issuer.
+      constexpr int QP = (NRP * 16 + kSoftmaxThreads - 1) / kSoftmaxThreads;
+      uint4 qval[QP];
+      auto q_load = [&](int item) {
         const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
         const __nv_bfloat16* qb = a.q + (long long)layer * a.q_ls + (long long)kvh * a.G * a.D;
         const int cpr = a.D >> 3;                        // 16-byte pieces per query row: 16, or 8 when D = 64
-        // every piece of a thread is loaded before the first is stored: one global round trip instead of up to eight
-        constexpr int QP = (NRP * 16 + kSoftmaxThreads - 1) / kSoftmaxThreads;
-        uint4 val[QP];
 #pragma unroll
         for (int k = 0; k < QP; ++k) {
           const int idx = st + k * kSoftmaxThreads;
           if (idx < a.rows * cpr) {
             const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
             const int r = (int)(((uint32_t)row * a.g_magic) >> 16), gq = row - r * a.G;
-            val[k] = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
+            qval[k] = *reinterpret_cast<const uint4*>(qb + ((long long)r * a.Hq + gq) * a.D + c * 8);
           }
         }
+      };
+      auto q_store = [&]() {
+        const int cpr = a.D >> 3;
 #pragma unroll
         for (int k = 0; k < QP; ++k) {
           const int idx = st + k * kSoftmaxThreads;
           if (idx < a.rows * cpr) {
             const int row = a.D == 128 ? idx >> 4 : idx >> 3, c = idx & (cpr - 1);
-            *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val[k];
+            *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = qval[k];
           }
         }
         fence_proxy_async();
         mbar_arrive(bar(Q_READY));
       };
-      stage_q((int)(f_begin / Tt));
+      q_load((int)(f_begin / Tt));
+      q_store();
       if (st == 0) PHASE(2)
       for (long long f = f_begin; f < f_end; ++seg) {
         const int item = (int)(f / Tt), tile0 = (int)(f - (long long)item * Tt);
@@ -718,10 +723,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // Both groups have read the scores of their last tiles, so every score MMA of this segment is done and Q is
         // free: the next item's Q goes in now, and the issuer starts that segment's score MMAs while the epilogue
         // below drains this segment's accumulators.
-        if (seg_end < f_end) stage_q(item + 1);
+        if (seg_end < f_end) q_load(item + 1);             // in flight during the wait below
         // ---- segment epilogue: this group's partial O (fp32), and (m, l) per row ----
         ok &= mbar_wait(bar(O_FULL), seg & 1, s_abort);
         tc_fence_after();
+        if (seg_end < f_end) q_store();
         const long long slot = ((long long)blockIdx.x * a.seg_max + (item - item_first)) * 2 + g;
         float* po = a.part_o + slot * NRP * 128;
         const bool has_tiles = i_first < n;
