@@ -35,6 +35,12 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// Programmatic dependent launch: a kernel lets the next one in the stream start its CTAs early
+// (pdl_launch_dependents), and that one blocks in pdl_wait until the kernels before it have completed and their
+// writes are visible.  Everything a kernel reads that an earlier kernel of the call wrote comes after pdl_wait.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 constexpr int kSimRowsPerCta = 8;      // text rows per CTA of the text pass (one per warp)
 
 // Text pass, one read of the text rows from HBM: a CTA takes 8 consecutive rows; each warp computes 1 / |X_j| of
@@ -42,6 +48,7 @@ constexpr int kSimRowsPerCta = 8;      // text rows per CTA of the text pass (on
 // (the rows come back from L1 / L2) and writes one partial of u.  Fixed order everywhere: deterministic.
 __global__ void __launch_bounds__(256) sim_text_kernel(const SimArgs a) {
   __shared__ float s_inv[kSimRowsPerCta];
+  pdl_launch_dependents();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int r0 = blockIdx.x * kSimRowsPerCta;
   for (int k = warp; k < kSimRowsPerCta; k += 8) {
@@ -63,11 +70,17 @@ __global__ void __launch_bounds__(256) sim_text_kernel(const SimArgs a) {
           for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
         }
       }
-      for (; c < n4; c += 32) {
-        float f[8];
-        unpack8(__ldg(src + c), f);
+      if (c < n4) {                                         // the remainder as one batch too (zeros add nothing)
+        uint4 v[7];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+        for (int i = 0; i < 7; ++i) v[i] = c + i * 32 < n4 ? __ldg(src + c + i * 32) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int i = 0; i < 7; ++i) {
+          float f[8];
+          unpack8(v[i], f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+        }
       }
     }
     acc = warp_sum(acc);
@@ -100,6 +113,8 @@ __global__ void __launch_bounds__(256) sim_text_kernel(const SimArgs a) {
 // loads in flight each, and their sums are merged in warp order.  The order is fixed: deterministic.
 __global__ void __launch_bounds__(256) sim_text_reduce_kernel(const SimArgs a, int n_part) {
   __shared__ float s_sum[8][32];
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = blockIdx.x * 32 + lane;
   float sacc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -127,9 +142,10 @@ __global__ void __launch_bounds__(256) sim_text_reduce_kernel(const SimArgs a, i
 // sim_i = (V_i . u) / |V_i|: u staged in shared memory, one warp per visual row, 16-byte loads.
 __global__ void __launch_bounds__(256) sim_visual_kernel(const SimArgs a) {
   extern __shared__ float s_u[];
-  for (int c = threadIdx.x; c < a.d; c += 256) s_u[c] = a.u[c];
-  __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  pdl_wait();
+  for (int c = threadIdx.x; c < a.d; c += 256) s_u[c] = __ldcg(a.u + c);
+  __syncthreads();
   for (int row = blockIdx.x * 8 + warp; row < a.m; row += gridDim.x * 8) {
     const uint4* src = reinterpret_cast<const uint4*>(a.h + (long long)(a.vis_start + row) * a.row_stride);
     float dot = 0.f, nrm = 0.f;
@@ -177,15 +193,30 @@ pvlm_status launch_similarity(const pvlm_similarity_params& p, cudaStream_t s) {
   a.u_part = (float*)ws;
   a.u = (float*)(ws + align_up((size_t)parts * p.d * 4, 256));
   a.inv_norm = nullptr;
+  // the second and third kernel are launched as programmatic dependents of the one before (see pdl_wait)
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(256);
+  cfg.stream = s;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaSuccess;
   if (p.n > 0) sim_text_kernel<<<parts, 256, 0, s>>>(a);
-  sim_text_reduce_kernel<<<ceil_div(p.d, 32), 256, 0, s>>>(a, p.n > 0 ? parts : 0);
-  if (p.m > 0) {
+  cfg.gridDim = dim3(ceil_div(p.d, 32));
+  cfg.dynamicSmemBytes = 0;
+  e = cudaLaunchKernelEx(&cfg, sim_text_reduce_kernel, a, p.n > 0 ? parts : 0);
+  if (e == cudaSuccess && p.m > 0) {
     int blocks = ceil_div(p.m, 8);
     if (blocks > kNumSMs * 16) blocks = kNumSMs * 16;
     const int smem = p.d * 4;
-    cudaFuncSetAttribute(sim_visual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    sim_visual_kernel<<<blocks, 256, smem, s>>>(a);
+    e = cudaFuncSetAttribute(sim_visual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cfg.gridDim = dim3(blocks);
+    cfg.dynamicSmemBytes = smem;
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, sim_visual_kernel, a);
   }
+  if (e != cudaSuccess) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   return check_launch();
 }
 
