@@ -88,7 +88,9 @@ class ClockSampler:
         self.f.close()
         os.unlink(self.f.name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w": statistics.median(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w": statistics.median(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons),
+                "power_note": "power.draw is nvidia-smi's moving average over about a second, so a timed region "
+                              "shorter than that reads low; sw_power_cap is the instantaneous flag"}
 
 
 # --------------------------------------------------------------------------------------
@@ -628,7 +630,7 @@ def cpu_baseline(cfg, w=None, gpu=None):
     The first sampled layer is the one the bench's mass row and o come from, so the timed GPU results of that layer
     (and the accept outcome) are compared with the oracle's here: `parity` in the returned object."""
     from paper_2603_19610_b200 import workloads as wl
-    n_sample = min(cfg.n_layers, 4) if cfg.n_layers > 1 else 1
+    n_sample = min(cfg.n_layers, 16)
     acc_inputs = wl.accept_inputs(cfg)
     heads = list(range(cfg.Hq))
     ta = tp = tc = 0.0
@@ -664,12 +666,13 @@ def run_reference(args):
     attn_inputs = wl.attn_layer(cfg, cfg.cur_layer)
     acc_inputs = wl.accept_inputs(cfg)
     # The per-step sample is sized so that the whole run (K + W steps) ends within a few minutes: one calibration
-    # step on a single query head, then as many heads (1..4) as a budget of ~150 s over all steps allows.
+    # step on every query head of the layer; if a budget of ~150 s over all steps does not allow that, proportionally
+    # fewer heads (the scaling to all heads then overstates the step, since converting K and V to fp64 is paid per call).
     t_cal = time.perf_counter()
-    oracle_sample_step(cfg, attn_inputs, acc_inputs, [0])
+    oracle_sample_step(cfg, attn_inputs, acc_inputs, list(range(cfg.Hq)))
     t_cal = time.perf_counter() - t_cal
     budget = 150.0 / max(1, args.steps + args.warmup)
-    n_heads = max(1, min(cfg.Hq, 4, int(budget / max(t_cal, 1e-3))))
+    n_heads = cfg.Hq if t_cal <= budget else max(1, int(cfg.Hq * budget / t_cal))
     heads = list(range(n_heads))
     for _ in range(args.warmup):
         oracle_sample_step(cfg, attn_inputs, acc_inputs, heads)
