@@ -9,6 +9,13 @@
  *   - Calls are asynchronous on the CUDA stream passed as `void *stream`
  *     (a cudaStream_t; NULL = default stream).  The library never
  *     synchronises the stream or the device.
+ *   - Calls whose data pointers are all device pointers (pvlm_verify_attn,
+ *     pvlm_uvprune_select_gather, pvlm_uvprune_similarity, pvlm_spec_accept,
+ *     pvlm_acceptance_rate, and pvlm_verify_step without host buffers) allocate
+ *     nothing and read nothing back, so they may be issued on a stream that is
+ *     being captured into a CUDA graph; the graph then replays them on the
+ *     same buffers.  pvlm_parallel_decode and pvlm_verify_step with host
+ *     buffers read results on the host and cannot be captured.
  *   - Scratch memory is caller-provided: `workspace` must hold at least the
  *     number of bytes the matching *_workspace_bytes query returns for the
  *     same parameter struct, and be 256-byte aligned.  Workspace contents are

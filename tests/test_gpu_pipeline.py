@@ -230,3 +230,87 @@ def test_draft_and_verify_streams_run_concurrently_and_agree():
     torch.cuda.synchronize()
     assert torch.equal(o_c, o_s) and torch.equal(mass_c, mass_s) and torch.equal(lse_c, lse_s)
     assert torch.equal(od_c, od_s) and torch.equal(lsed_c, lsed_s)
+
+
+@pytest.mark.parametrize("cid", [0, 1])
+def test_the_three_calls_replay_from_a_cuda_graph(cid):
+    """pvlm_verify_attn -> pvlm_uvprune_select_gather -> pvlm_spec_accept on device-resident inputs
+    make no host round trip, so a stream capture records them; the replayed graph, fed new contents in
+    the same buffers, gives what the direct calls give, bit for bit, and matches the oracle."""
+    cfg = wl.CONFIGS[cid]
+    ref_in, cur_in = layers_for(cfg)
+    q = torch.stack([bf16_cuda(ref_in[0]), bf16_cuda(cur_in[0])])
+    k = torch.stack([bf16_cuda(ref_in[1]), bf16_cuda(cur_in[1])])
+    v = torch.stack([bf16_cuda(ref_in[2]), bf16_cuda(cur_in[2])])
+    tl, dl, tok, u = (torch.from_numpy(x).cuda() for x in wl.accept_inputs(cfg))
+
+    def run():
+        o, lse, mass = binding.verify_attn(q, k, v, cfg.n_ctx, want_mass=True, mass_layers=[0, 1])
+        kept, _, dk, dv = binding.uvprune_select_gather(mass[1], mass[0], 0, cfg.m, cfg.k_keep, k, v)
+        acc = binding.spec_accept(tl, dl, tok, u)
+        return o, lse, mass, kept, dk, dv, acc["n_accept"], acc["out_tokens"]
+
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):                       # warm-up: workspaces and function attributes exist before the capture
+        run()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        outs = run()
+    for rnd in range(2):
+        if rnd == 1:                                 # new contents, same buffers: the window rows of another seed, swapped logits
+            q2, k2, v2 = (bf16_cuda(x) for x in wl.make_qkv(cfg.Hq, cfg.Hkv, cfg.D, cfg.R, cfg.T, sink=True, seed=4242 + cid))
+            q[1].copy_(q2); k[1].copy_(k2); v[1].copy_(v2)
+            u.copy_(torch.flip(u, [0]))
+        for t in outs:
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        got = [t.clone() for t in outs]
+        want = run()
+        torch.cuda.synchronize()
+        for a, b in zip(got, want):
+            assert torch.equal(a, b)
+    # the second replay against the oracle
+    O, L, M = oracle_attn(bits_of(q[1]), bits_of(k[1]), bits_of(v[1]), cfg.n_ctx)
+    assert_o_close(got[0][1], O)
+    assert_rel_close(got[2][1].cpu().numpy(), M, what="mass")
+    r = oracle_accept(tl.cpu().numpy(), dl.cpu().numpy(), tok.cpu().numpy(), u.cpu().numpy())
+    assert int(got[6]) == r["n_accept"]
+
+
+def test_similarity_and_acceptance_rate_replay_from_a_cuda_graph():
+    """The hidden-state criterion (three kernels chained by programmatic dependent launch) and the acceptance-rate
+    pass are capturable too: a replay equals the direct calls bit for bit."""
+    dev = torch.device("cuda")
+    g0 = torch.Generator(device="cpu").manual_seed(31)
+    hidden = torch.randn((700 + 90, 1024), generator=g0).to(torch.bfloat16).to(dev)
+    N, V = 40, 3001
+    tl = torch.randn((N, V), generator=g0).mul_(3).to(dev)
+    dl = (tl.cpu() + 0.5 * torch.randn((N, V), generator=g0)).to(dev)
+    tok = torch.randint(0, V, (N,), generator=g0, dtype=torch.int32).to(dev)
+    u = torch.rand(N, generator=g0).to(dev)
+
+    def run():
+        sim = binding.uvprune_similarity(hidden, 0, 700, 700, 90)
+        r = binding.acceptance_rate(tl, dl, tok, u)
+        return sim, r["accepted"], r["n_accepted"], r["p_tok"], r["q_tok"]
+
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        run()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        outs = run()
+    hidden.copy_(torch.randn(hidden.shape, generator=g0).to(torch.bfloat16))
+    u.copy_(torch.rand(N, generator=g0))
+    for t in outs:
+        t.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    want = run()
+    torch.cuda.synchronize()
+    for a, b in zip(outs, want):
+        assert torch.equal(a, b)
+    assert float(outs[0].abs().max()) > 0
