@@ -501,7 +501,19 @@ def draft_stream_leg(cfg, dev, torch, binding, wl, Q, K, V, O, lse, mass, w, pp,
             for p in pd_full:
                 binding.verify_step(p, None, None, device=dev)
 
+    # the draft window as one CUDA graph (its twelve steps are 24 short launches: the launch-bound loop of the path)
+    torch.cuda.synchronize()
+    gd = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gd, stream=sD):
+        for p in pd_full:
+            binding.verify_step(p, None, None, device=dev)
+
+    def draft_graph():
+        with torch.cuda.stream(sD):
+            gd.replay()
+
     reps = 12
+    _, d_graph = timed(None, draft_graph, reps)
     v_alone, _ = timed(verify, None, reps)
     _, d_alone = timed(None, draft, reps)
     v_con, d_con = timed(verify, draft, reps)
@@ -514,7 +526,8 @@ def draft_stream_leg(cfg, dev, torch, binding, wl, Q, K, V, O, lse, mass, w, pp,
             "verify_step_us_alone": v_alone, "draft_window_us_alone": d_alone,
             "verify_step_us_concurrent": v_con, "draft_window_us_concurrent": d_con,
             "both_us_concurrent": max(v_con, d_con), "both_us_serial": v_alone + d_alone,
-            "verify_step_us_all_sms": v_full, "draft_window_us_all_sms": d_full, "both_us_serial_all_sms": v_full + d_full,
+            "verify_step_us_all_sms": v_full, "draft_window_us_all_sms": d_full, "draft_window_us_all_sms_graph_replay": d_graph,
+            "both_us_serial_all_sms": v_full + d_full,
             "note": "both streams share one GPU's HBM. both_us_serial runs the same SM-limited kernels one after the other; "
                     "both_us_serial_all_sms gives each side every SM, one after the other (the honest serial reference): side by "
                     "side still wins because the draft's twelve short decode steps are latency-bound on their own"}
