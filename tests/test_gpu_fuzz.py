@@ -1,0 +1,121 @@
+"""Seeded random-geometry sweeps of every call (GPU): the tensor-core attention against the mma.sync
+implementation over ragged shapes, CTA counts, both cache layouts and mass-layer subsets; selection,
+gather and the accept path against the CPU oracle.  PVLM_FUZZ_CASES scales the number of cases
+(default 60 per call; a few hundred take about a minute)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle.uvprune import gather_rows, score_fp32, select_topk
+from paper_2603_19610_b200 import binding
+from helpers import bits_of
+from test_gpu_accept import check_against_oracle
+from test_gpu_prune import gpu_select
+
+pytestmark = pytest.mark.gpu
+CASES = int(os.environ.get("PVLM_FUZZ_CASES", "60"))
+
+
+def test_attention_random_geometries(monkeypatch):
+    rng = np.random.default_rng(11)
+    for case in range(CASES):
+        D = int(rng.choice([64, 128]))
+        Hkv = int(rng.integers(1, 9))
+        G = int(rng.choice([1, 2, 3, 4, 5, 6, 7, 8, 12, 16]))
+        R = int(rng.integers(1, max(2, 128 // G + 1)))
+        n_ctx = int(rng.choice([0, 1, 2, 63, 64, 127, 128, 129, 255, 256, 257, 700, 2500, int(rng.integers(0, 9000))]))
+        L = int(rng.integers(1, 6))
+        ctas = int(rng.choice([0, 0, 1, 2, 5, 37, 148]))
+        head_major = bool(rng.integers(0, 2))
+        Hq, T = G * Hkv, n_ctx + R
+        g = torch.Generator(device="cuda")
+        g.manual_seed(case)
+        mk = lambda *sh: torch.randn(sh, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        q, k, v = mk(L, R, Hq, D), mk(L, T, Hkv, D), mk(L, T, Hkv, D)
+        if rng.integers(0, 3) == 0:                      # a sink-like first key now and then
+            k[:, 0] *= 4
+        if head_major:                                   # [layer][kv_head][token][D] storage behind the same view
+            k = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+            v = v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        ml = None
+        if L > 1 and rng.integers(0, 2):
+            ml = sorted(set(int(x) for x in rng.integers(0, L, size=2)))
+        monkeypatch.delenv("PVLM_ATTN_IMPL", raising=False)
+        if ctas:
+            monkeypatch.setenv("PVLM_TC_CTAS", str(ctas))
+        else:
+            monkeypatch.delenv("PVLM_TC_CTAS", raising=False)
+        o1, l1, m1 = binding.verify_attn(q, k, v, n_ctx, want_mass=True, check=True, mass_layers=ml)
+        monkeypatch.delenv("PVLM_TC_CTAS", raising=False)
+        monkeypatch.setenv("PVLM_ATTN_IMPL", "mma")
+        o2, l2, m2 = binding.verify_attn(q, k, v, n_ctx, want_mass=True, mass_layers=ml)
+        torch.cuda.synchronize()
+        tag = (case, L, Hq, Hkv, D, n_ctx, R, ctas, head_major, ml)
+        err = (o1.float() - o2.float()).abs()
+        assert bool(torch.isfinite(o1.float()).all()), tag
+        assert bool((err <= 1e-2 + 2e-2 * o2.float().abs()).all()), tag
+        assert float((l1 - l2).abs().max()) <= 1e-4, tag
+        assert bool(((m1 - m2).abs() <= 1e-4 * m2.abs() + 1e-30).all()), tag
+
+
+def test_select_random_sizes_and_score_distributions():
+    rng = np.random.default_rng(5)
+    for case in range(CASES):
+        m = int(rng.choice([1, 2, 31, 32, 33, 1000, 4095, 4096, 4097, int(rng.integers(1, 200000))]))
+        k = int(rng.choice([0, 1, m, max(0, m - 1), int(rng.integers(0, m + 1))]))
+        v0 = int(rng.integers(0, 40))
+        T = v0 + m + int(rng.integers(0, 20))
+        kind = int(rng.integers(0, 4))
+        if kind == 0:
+            cur = rng.random(T).astype(np.float32)
+        elif kind == 1:
+            cur = (np.round(rng.standard_normal(T) * 4) / 4).astype(np.float32)        # heavy ties
+        elif kind == 2:
+            cur = np.full(T, 0.5, dtype=np.float32)                                    # all equal
+        else:
+            cur = (rng.standard_normal(T) * 10.0 ** rng.integers(-30, 30)).astype(np.float32)
+        ref = rng.random(T).astype(np.float32) if rng.integers(0, 2) else None
+        kept, score = gpu_select(cur, ref, v0, m, k)
+        s_ref = score_fp32(cur, ref, v0, m)
+        tag = (case, m, k, v0, kind, ref is not None)
+        assert (score.view(np.uint32) == s_ref.view(np.uint32)).all(), tag
+        assert (kept == select_topk(s_ref, k)).all(), tag
+
+
+def test_gather_random_shapes():
+    rng = np.random.default_rng(6)
+    for case in range(max(10, CASES // 3)):
+        L, Hkv, D = int(rng.integers(1, 5)), int(rng.choice([1, 2, 4, 8])), int(rng.choice([64, 128]))
+        S = int(rng.integers(2, 3000))
+        v0 = int(rng.integers(0, S))
+        m = int(rng.integers(0, S - v0 + 1))
+        k = int(rng.integers(0, m + 1))
+        kb = rng.integers(0, 65536, size=(L, S, Hkv, D), dtype=np.uint16)
+        vb = rng.integers(0, 65536, size=(L, S, Hkv, D), dtype=np.uint16)
+        mass = rng.random(S).astype(np.float32)
+        to_dev = lambda b: torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).cuda()
+        kept, _, dk, dv = binding.uvprune_select_gather(torch.from_numpy(mass).cuda(), None, v0, m, k, to_dev(kb), to_dev(vb))
+        torch.cuda.synchronize()
+        idx = kept.cpu().numpy()
+        tag = (case, L, S, Hkv, D, v0, m, k)
+        assert (idx == select_topk(mass[v0:v0 + m], k)).all(), tag
+        assert bits_of(dk).tobytes() == gather_rows(kb, v0, m, idx).tobytes(), tag
+        assert bits_of(dv).tobytes() == gather_rows(vb, v0, m, idx).tobytes(), tag
+
+
+def test_accept_random_vocab_window_and_temperature():
+    rng = np.random.default_rng(8)
+    for case in range(CASES):
+        V = int(rng.choice([1, 2, 3, 17, 255, 256, 257, 1000, 4096, 5000, int(rng.integers(1, 40000))]))
+        gamma = int(rng.integers(1, 65 if V < 3000 else 17))
+        sig = float(rng.choice([0.0, 0.1, 0.5, 2.0]))
+        temp = float(rng.choice([1.0, 1.0, 0.7, 1.5]))
+        tl = (rng.standard_normal((gamma + 1, V)) * 3).astype(np.float32)
+        dl = (tl[:gamma] + sig * rng.standard_normal((gamma, V))).astype(np.float32)
+        tok = rng.integers(0, V, size=gamma).astype(np.int32)
+        if rng.integers(0, 2):                           # the draft row's most likely token: usually accepted
+            tok = dl.argmax(1).astype(np.int32)
+        u = rng.random(gamma + 1).astype(np.float32)
+        check_against_oracle(tl, dl, tok, u, temp)
