@@ -143,7 +143,7 @@ typedef struct {
   int *kept_idx;         /* int32 [k] out                                                      */
   float *score;          /* fp32 [m] out; nullable                                             */
   const void *src_k, *src_v; /* [n_layers][src_len][row_bytes]; both NULL => select only      */
-  void *dst_k, *dst_v;       /* [n_layers][src_len - m + k][row_bytes]                         */
+  void *dst_k, *dst_v;       /* [n_layers][src_len - m + k][row_bytes]; may be NULL if that is 0 rows */
   int n_layers, src_len;
   long long row_bytes;
   long long src_layer_stride_bytes, dst_layer_stride_bytes;

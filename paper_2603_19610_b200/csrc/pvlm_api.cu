@@ -122,12 +122,13 @@ static pvlm_status validate_prune(const pvlm_prune_params* p) {
   if (p->k > 0 && !p->kept_idx) return PVLM_ERR_INVALID_ARG;
   const bool gather = p->src_k || p->src_v || p->dst_k || p->dst_v;
   if (gather) {
-    if (!p->src_k || !p->src_v || !p->dst_k || !p->dst_v) return PVLM_ERR_INVALID_ARG;
+    if (!p->src_k || !p->src_v) return PVLM_ERR_INVALID_ARG;
     if (p->n_layers < 1 || p->row_bytes <= 0 || p->src_len < p->vis_start + p->m) return PVLM_ERR_INVALID_ARG;
+    const long long dst_len = (long long)p->src_len - p->m + p->k;
+    if (dst_len > 0 && (!p->dst_k || !p->dst_v)) return PVLM_ERR_INVALID_ARG;     // an empty compacted cache needs no storage
     if (p->row_bytes % 16) return PVLM_ERR_UNSUPPORTED;
     if (!aligned(p->src_k, 16) || !aligned(p->src_v, 16) || !aligned(p->dst_k, 16) || !aligned(p->dst_v, 16))
       return PVLM_ERR_INVALID_ARG;
-    const long long dst_len = (long long)p->src_len - p->m + p->k;
     if (p->n_layers > 1) {
       if (p->src_layer_stride_bytes < (long long)p->src_len * p->row_bytes || p->src_layer_stride_bytes % 16) return PVLM_ERR_INVALID_ARG;
       if (p->dst_layer_stride_bytes < dst_len * p->row_bytes || p->dst_layer_stride_bytes % 16) return PVLM_ERR_INVALID_ARG;

@@ -119,3 +119,36 @@ def test_accept_random_vocab_window_and_temperature():
             tok = dl.argmax(1).astype(np.int32)
         u = rng.random(gamma + 1).astype(np.float32)
         check_against_oracle(tl, dl, tok, u, temp)
+
+
+def test_step_overlap_mode_random_gather_splits():
+    """pvlm_verify_step in overlap mode (rows outside the visual span copied on the second stream, selected rows on
+    the main one) against the one-call select + gather: empty spans on either side, k = 0 and k = m included."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(9)
+    cs, ea, eb = torch.cuda.Stream(), torch.cuda.Event(), torch.cuda.Event()
+    ea.record()
+    eb.record()
+    torch.cuda.synchronize()
+    for case in range(max(10, CASES // 2)):
+        L, Hkv, D = int(rng.integers(1, 4)), int(rng.choice([1, 2, 4, 8])), int(rng.choice([64, 128]))
+        S = int(rng.integers(2, 2500))
+        v0 = int(rng.choice([0, 0, int(rng.integers(0, S))]))
+        m = int(rng.choice([S - v0, int(rng.integers(0, S - v0 + 1))]))
+        k = int(rng.choice([0, m, int(rng.integers(0, m + 1))]))
+        g = torch.Generator(device="cuda")
+        g.manual_seed(1000 + case)
+        src_k = torch.randn((L, S, Hkv, D), generator=g, device=dev).to(torch.bfloat16)
+        src_v = torch.randn((L, S, Hkv, D), generator=g, device=dev).to(torch.bfloat16)
+        cur = torch.rand(S, generator=g, device=dev)
+        ref = torch.rand(S, generator=g, device=dev)
+        kept_e, _, dk_e, dv_e = binding.uvprune_select_gather(cur, ref, v0, m, k, src_k, src_v)
+        kept = torch.full((max(k, 1),), -7, dtype=torch.int32, device=dev)
+        dk = torch.zeros((L, S - m + k, Hkv, D), dtype=torch.bfloat16, device=dev)
+        dv = torch.zeros_like(dk)
+        pp = binding.prune_params(cur, ref, v0, m, k, kept, None, src_k, src_v, dk, dv)
+        binding.verify_step(None, pp, None, device=dev, overlap=(cs, ea, eb))
+        torch.cuda.current_stream().synchronize()
+        tag = (case, L, S, Hkv, D, v0, m, k)
+        assert torch.equal(kept[:k], kept_e[:k]), tag
+        assert torch.equal(dk, dk_e) and torch.equal(dv, dv_e), tag
