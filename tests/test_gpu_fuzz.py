@@ -8,11 +8,15 @@ import numpy as np
 import pytest
 import torch
 
+from oracle.pipeline import parallel_decode as oracle_decode
 from oracle.uvprune import gather_rows, score_fp32, select_topk
-from paper_2603_19610_b200 import binding
+from paper_2603_19610_b200 import binding, workloads as wl
 from helpers import bits_of
 from test_gpu_accept import check_against_oracle
+from test_gpu_decode import gpu_decode, log_rows, make_case
 from test_gpu_prune import gpu_select
+from test_gpu_rate import run_case as rate_case
+from test_gpu_similarity import check as similarity_check
 
 pytestmark = pytest.mark.gpu
 CASES = int(os.environ.get("PVLM_FUZZ_CASES", "60"))
@@ -152,3 +156,43 @@ def test_step_overlap_mode_random_gather_splits():
         tag = (case, L, S, Hkv, D, v0, m, k)
         assert torch.equal(kept[:k], kept_e[:k]), tag
         assert torch.equal(dk, dk_e) and torch.equal(dv, dv_e), tag
+
+
+def test_parallel_decode_random_windows_vocabularies_and_temperatures():
+    rng = np.random.default_rng(2)
+    for case in range(CASES):
+        V = int(rng.choice([2, 3, 17, 50, 257, 1000, 4099, int(rng.integers(2, 20000))]))
+        K, gamma = int(rng.integers(1, 60)), int(rng.integers(1, 17))
+        sigma = float(rng.choice([0.0, 0.2, 0.6, 1.5]))
+        temp = float(rng.choice([1.0, 1.0, 0.8]))
+        tl, dl, ud, ua, ur = make_case(V, K, gamma, sigma, 100 + case)
+        ref = oracle_decode(tl, dl, gamma, K, ud, ua, ur, temp)
+        for serial in (False, True):
+            out = gpu_decode(tl, dl, gamma, K, ud, ua, ur, serial=serial, temperature=temp)
+            tag = (case, V, K, gamma, sigma, temp, serial)
+            assert out["rounds"] == ref["rounds"], tag
+            assert out["log"].tolist() == log_rows(ref["log"]), tag
+            assert (out["tokens"].numpy() == ref["tokens"]).all(), tag
+
+
+def test_acceptance_rate_random_sizes_and_strides():
+    rng = np.random.default_rng(3)
+    for case in range(CASES):
+        N = int(rng.choice([0, 1, 2, 33, 100, int(rng.integers(1, 600))]))
+        V = int(rng.choice([1, 2, 17, 255, 256, 1000, 4099, int(rng.integers(1, 30000))]))
+        rate_case(N, V, float(rng.choice([0.0, 0.3, 1.0])), 500 + case, float(rng.choice([1.0, 0.7, 1.3])),
+                  int(rng.choice([0, 0, 1, 2, 4])))
+
+
+def test_similarity_random_shapes():
+    rng = np.random.default_rng(4)
+    for case in range(CASES):
+        m = int(rng.choice([1, 7, 8, 9, 100, int(rng.integers(1, 3000))]))
+        n = int(rng.choice([0, 1, 7, 8, 9, 17, int(rng.integers(1, 600))]))
+        d = int(rng.choice([8, 16, 256, 264, 1000, 2560, 2568, 3584, 5120, 8192]))
+        v0 = int(rng.integers(0, 5))
+        h = rng.standard_normal((v0 + m + n + 2, d)).astype(np.float32)
+        h[v0 + m:] += 0.3                                # text rows share a direction
+        if m > 2 and rng.integers(0, 4) == 0:
+            h[v0 + 1] = 0                                # a zero visual row
+        similarity_check(wl.f32_to_bf16_bits(h), v0, m, v0 + m, n)
