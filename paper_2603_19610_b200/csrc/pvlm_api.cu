@@ -63,11 +63,11 @@ size_t pvlm_verify_attn_workspace_bytes(const pvlm_attn_params* p) {
   return plan.total;
 }
 
-pvlm_status pvlm_verify_attn(const pvlm_attn_params* p, void* stream) {
+// Every host-side check of an attention call; fills the plan.  Nothing is launched.
+static pvlm_status validate_attn(const pvlm_attn_params* p, AttnPlan& plan) {
   if (!p) return PVLM_ERR_INVALID_ARG;
   if (p->n_layers < 1 || p->R < 1 || p->Hq < 1 || p->Hkv < 1 || p->D < 1 || p->n_ctx < 0) return PVLM_ERR_INVALID_ARG;
   if (!p->q || !p->k || !p->v || !p->o) return PVLM_ERR_INVALID_ARG;
-  AttnPlan plan;
   if (!make_attn_plan(*p, plan)) return PVLM_ERR_UNSUPPORTED;
   if (!aligned(p->q, 16) || !aligned(p->k, 16) || !aligned(p->v, 16) || !aligned(p->o, 16)) return PVLM_ERR_INVALID_ARG;
   if (p->kv_head_stride < p->D || p->kv_head_stride % 8) return PVLM_ERR_INVALID_ARG;
@@ -88,8 +88,13 @@ pvlm_status pvlm_verify_attn(const pvlm_attn_params* p, void* stream) {
   }
   if (p->n_layers > 65535 || p->Hkv > 65535) return PVLM_ERR_UNSUPPORTED;
   if (p->max_ctas < 0) return PVLM_ERR_INVALID_ARG;
-  const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, plan.total);
-  if (w != PVLM_OK) return w;
+  return check_ws(p->workspace, p->workspace_bytes, plan.total);
+}
+
+pvlm_status pvlm_verify_attn(const pvlm_attn_params* p, void* stream) {
+  AttnPlan plan;
+  const pvlm_status v = validate_attn(p, plan);
+  if (v != PVLM_OK) return v;
   return launch_verify_attn(*p, plan, (cudaStream_t)stream);
 }
 
@@ -169,12 +174,12 @@ size_t pvlm_spec_accept_workspace_bytes(const pvlm_accept_params* p) {
   return plan.total;
 }
 
-pvlm_status pvlm_spec_accept(const pvlm_accept_params* p, void* stream) {
+// Every host-side check of an accept call; fills the plan.  Nothing is launched.
+static pvlm_status validate_accept(const pvlm_accept_params* p, AcceptPlan& plan) {
   if (!p) return PVLM_ERR_INVALID_ARG;
   if (p->gamma < 0 || p->V < 1 || p->batch < 1) return PVLM_ERR_INVALID_ARG;
   if (!p->target_logits || !p->uniforms || !p->n_accept || !p->out_tokens) return PVLM_ERR_INVALID_ARG;
   if (p->gamma > 0 && (!p->draft_logits || !p->draft_tokens)) return PVLM_ERR_INVALID_ARG;
-  AcceptPlan plan;
   if (!make_accept_plan(*p, plan)) return PVLM_ERR_UNSUPPORTED;
   if (p->batch > 65535) return PVLM_ERR_UNSUPPORTED;
   if (!aligned(p->target_logits, 4) || !aligned(p->draft_logits, 4)) return PVLM_ERR_INVALID_ARG;
@@ -185,8 +190,13 @@ pvlm_status pvlm_spec_accept(const pvlm_accept_params* p, void* stream) {
     if (p->draft_batch_stride != 0 && (p->draft_batch_stride < (long long)p->gamma * p->draft_row_stride)) return PVLM_ERR_INVALID_ARG;
   }
   if (p->temperature < 0.f) return PVLM_ERR_INVALID_ARG;
-  const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, plan.total);
-  if (w != PVLM_OK) return w;
+  return check_ws(p->workspace, p->workspace_bytes, plan.total);
+}
+
+pvlm_status pvlm_spec_accept(const pvlm_accept_params* p, void* stream) {
+  AcceptPlan plan;
+  const pvlm_status v = validate_accept(p, plan);
+  if (v != PVLM_OK) return v;
   return launch_spec_accept(*p, plan, (cudaStream_t)stream);
 }
 
@@ -201,13 +211,38 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
   const pvlm_accept_params& c = p->accept;
   cudaError_t e = cudaSuccess;
   auto ok = [&]() { return e == cudaSuccess; };
+  // ---- every argument check of the stages and the copies, before anything is queued on either stream ----
+  if (p->run_attn) {
+    AttnPlan plan;
+    const pvlm_status va = validate_attn(&a, plan);
+    if (va != PVLM_OK) return va;
+  }
+  if (p->run_attn && (p->h_k_window || p->h_v_window)) {
+    const bool token_major = a.kv_head_stride == a.D && a.kv_token_stride == (long long)a.Hkv * a.D;
+    const bool head_major = a.kv_token_stride == a.D && a.kv_head_stride >= (long long)(a.n_ctx + a.R) * a.D &&
+                            (a.n_layers == 1 || a.kv_layer_stride == (long long)a.Hkv * a.kv_head_stride);
+    if (!token_major && !head_major) return PVLM_ERR_UNSUPPORTED;
+  }
+  if (p->run_accept) {
+    AcceptPlan plan;
+    const pvlm_status vc = validate_accept(&c, plan);
+    if (vc != PVLM_OK) return vc;
+    if (p->h_target_logits || p->h_draft_logits) {
+      if (c.target_row_stride != c.V || c.draft_row_stride != c.V) return PVLM_ERR_UNSUPPORTED;
+      if (c.batch > 1 && (c.target_batch_stride != (long long)(c.gamma + 1) * c.V ||
+                          c.draft_batch_stride != (long long)c.gamma * c.V)) return PVLM_ERR_UNSUPPORTED;
+    }
+  }
+  if (p->run_prune) {
+    const pvlm_status vp = validate_prune(&p->prune);
+    if (vp != PVLM_OK) return vp;
+  }
   // ---- host -> device: this step's inputs ----
   if (overlap) {                       // the copy stream starts after whatever is already queued on `stream`
     e = cudaEventRecord(ea, s);
     if (ok()) e = cudaStreamWaitEvent(cs, ea, 0);
   }
   if (p->run_attn) {
-    if (a.n_layers < 1 || a.R < 1 || a.Hq < 1 || a.Hkv < 1 || a.D < 1 || a.n_ctx < 0) return PVLM_ERR_INVALID_ARG;
     const size_t q_layer = (size_t)a.R * a.Hq * a.D * 2;
     if (p->h_q && ok())
       e = cudaMemcpy2DAsync(const_cast<void*>(a.q), (size_t)a.q_layer_stride * 2, p->h_q, q_layer, q_layer, a.n_layers,
@@ -222,12 +257,10 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
         width = (size_t)a.R * a.Hkv * a.D * 2;
         pitch = a.n_layers > 1 ? (size_t)a.kv_layer_stride * 2 : width;
         height = a.n_layers;
-      } else if (head_major) {             // host [n_layers][Hkv][R][D]: one piece of R rows per (layer, KV head)
+      } else {                             // head-major (checked above); host [n_layers][Hkv][R][D]: one piece of R rows per (layer, KV head)
         width = (size_t)a.R * a.D * 2;
         pitch = (size_t)a.kv_head_stride * 2;
         height = a.n_layers * a.Hkv;
-      } else {
-        return PVLM_ERR_UNSUPPORTED;
       }
       if (p->h_k_window && ok())
         e = cudaMemcpy2DAsync((char*)const_cast<void*>(a.k) + row0, pitch, p->h_k_window, width, width, height,
@@ -243,12 +276,6 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     if (ok()) e = cudaStreamWaitEvent(cs, eb, 0);
   }
   if (p->run_accept) {
-    if (c.gamma < 0 || c.V < 1 || c.batch < 1) return PVLM_ERR_INVALID_ARG;
-    if (p->h_target_logits || p->h_draft_logits) {
-      if (c.target_row_stride != c.V || c.draft_row_stride != c.V) return PVLM_ERR_UNSUPPORTED;
-      if (c.batch > 1 && (c.target_batch_stride != (long long)(c.gamma + 1) * c.V ||
-                          c.draft_batch_stride != (long long)c.gamma * c.V)) return PVLM_ERR_UNSUPPORTED;
-    }
     const size_t B = (size_t)c.batch;
     if (p->h_target_logits && ok())
       e = cudaMemcpyAsync(const_cast<float*>(c.target_logits), p->h_target_logits, B * (c.gamma + 1) * c.V * 4, cudaMemcpyHostToDevice, cs);
@@ -269,7 +296,6 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
   pvlm_status st;
   const bool accept_on_side = overlap && p->run_accept;
   const bool split_gather = overlap && p->run_prune && p->prune.src_k;
-  if (split_gather && (st = validate_prune(&p->prune)) != PVLM_OK) return st;
   if (p->run_attn) {
     if (accept_on_side || split_gather) set_after_main_event(eb);
     st = pvlm_verify_attn(&p->attn, stream);

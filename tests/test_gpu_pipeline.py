@@ -314,3 +314,31 @@ def test_similarity_and_acceptance_rate_replay_from_a_cuda_graph():
     for a, b in zip(outs, want):
         assert torch.equal(a, b)
     assert float(outs[0].abs().max()) > 0
+
+
+def test_step_call_rejects_bad_arguments_before_queuing_anything():
+    """A bad argument in any stage of pvlm_verify_step is reported before the call touches either stream:
+    the second stream is not left waiting on a half-built step, and the next (valid) call is unaffected."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(5)
+    L, S, Hkv, D, v0, m, k = 2, 500, 2, 64, 3, 400, 100
+    src_k = torch.randn((L, S, Hkv, D), device=dev).to(torch.bfloat16)
+    src_v = torch.randn((L, S, Hkv, D), device=dev).to(torch.bfloat16)
+    cur = torch.from_numpy(rng.random(S).astype(np.float32)).to(dev)
+    kept_e, _, dk_e, dv_e = binding.uvprune_select_gather(cur, None, v0, m, k, src_k, src_v)
+    kept = torch.zeros(k, dtype=torch.int32, device=dev)
+    dk = torch.zeros((L, S - m + k, Hkv, D), dtype=torch.bfloat16, device=dev)
+    dv = torch.zeros_like(dk)
+    pp = binding.prune_params(cur, None, v0, m, k, kept, None, src_k, src_v, dk, dv)
+    cs, ea, eb = torch.cuda.Stream(), torch.cuda.Event(), torch.cuda.Event()
+    ea.record(); eb.record()
+    torch.cuda.synchronize()
+    pp.k = m + 1                                              # more kept tokens than visual tokens
+    with pytest.raises(binding.PvlmError) as err:
+        binding.verify_step(None, pp, None, device=dev, overlap=(cs, ea, eb))
+    assert "INVALID_ARG" in str(err.value)
+    assert cs.query() and torch.cuda.current_stream().query()  # nothing was queued
+    pp.k = k
+    binding.verify_step(None, pp, None, device=dev, overlap=(cs, ea, eb))
+    torch.cuda.current_stream().synchronize()
+    assert torch.equal(kept, kept_e) and torch.equal(dk, dk_e) and torch.equal(dv, dv_e)
