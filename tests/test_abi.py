@@ -90,6 +90,22 @@ def test_workspace_queries_and_argument_errors_need_no_gpu():
     assert L.pvlm_uvprune_workspace_bytes(C.byref(u)) >= 400
     assert L.pvlm_uvprune_select_gather(C.byref(u), None) == 1          # no mass pointer
 
+    # the step call checks every stage before it queues anything (so this needs no GPU either)
+    sp = binding.StepParams()
+    assert L.pvlm_verify_step(None, None) == 1
+    sp.run_prune = 1
+    sp.prune.m, sp.prune.k = 100, 101
+    assert L.pvlm_verify_step(C.byref(sp), None) == 1                   # k > m in the prune stage
+    sp.run_prune, sp.run_accept = 0, 1
+    sp.accept.batch, sp.accept.gamma, sp.accept.V = 1, 12, 152064
+    assert L.pvlm_verify_step(C.byref(sp), None) == 1                   # accept stage without logits
+    sp.run_accept, sp.run_attn = 0, 1
+    sp.attn.n_layers, sp.attn.R, sp.attn.Hq, sp.attn.Hkv, sp.attn.D, sp.attn.n_ctx = 1, 13, 40, 8, 96, 1000
+    sp.attn.q = sp.attn.k = sp.attn.v = sp.attn.o = 4096
+    assert L.pvlm_verify_step(C.byref(sp), None) == 2                   # D = 96 in the attention stage
+    sp.copy_stream = 1                                                   # overlap mode needs the stream AND both events
+    assert L.pvlm_verify_step(C.byref(sp), None) == 1
+
 
 def test_no_cpu_fallback():
     import torch
