@@ -290,3 +290,37 @@ def test_tensor_core_and_mma_sync_paths_agree_on_random_shapes(monkeypatch):
         assert bool((err <= 1e-2 + 2e-2 * o2.float().abs()).all()), tag
         assert float((l1 - l2).abs().max()) <= 1e-4, tag
         assert bool(((m1 - m2).abs() <= 1e-4 * m2.abs() + 1e-30).all()), tag
+
+
+def test_config2_all_64_layers_in_the_bench_launch_configuration():
+    """The launch bench.py times: all 64 layers of config 2 in ONE call (head-major cache, mass on the reference and
+    the current layer, 889 tiles and 3.5 items per persistent CTA).  Three layers hold the host-generated data of the
+    workload recipe and are checked in full against the oracle; the others are device-drawn filler of the same shape."""
+    cfg = wl.CONFIGS[2]
+    L, T, R = cfg.n_layers, cfg.T, cfg.R
+    dev = torch.device("cuda")
+    g = torch.Generator(device=dev)
+    g.manual_seed(99)
+    k_base = torch.empty((L, cfg.Hkv, T, cfg.D), dtype=torch.bfloat16, device=dev)
+    v_base = torch.empty_like(k_base)
+    q = torch.empty((L, R, cfg.Hq, cfg.D), dtype=torch.bfloat16, device=dev)
+    for l in range(L):
+        k_base[l].copy_(torch.randn((cfg.Hkv, T, cfg.D), generator=g, device=dev))
+        v_base[l].copy_(torch.randn((cfg.Hkv, T, cfg.D), generator=g, device=dev))
+        q[l].copy_(torch.randn((R, cfg.Hq, cfg.D), generator=g, device=dev))
+    k, v = k_base.permute(0, 2, 1, 3), v_base.permute(0, 2, 1, 3)          # the [layer][token][kv_head][D] view
+    checked = {l: wl.attn_layer(cfg, l) for l in (cfg.ref_layer, cfg.cur_layer, L - 1)}
+    for l, (qb, kb, vb) in checked.items():
+        q[l].copy_(bf16_cuda(qb)); k[l].copy_(bf16_cuda(kb)); v[l].copy_(bf16_cuda(vb))
+    mass_layers = [cfg.ref_layer, cfg.cur_layer]
+    o, lse, mass = binding.verify_attn(q, k, v, cfg.n_ctx, want_mass=True, mass_layers=mass_layers, check=True)
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(o.float()).all()) and bool(torch.isfinite(lse).all())
+    for l, (qb, kb, vb) in checked.items():
+        O, Lr, M = oracle_attn(qb, kb, vb, cfg.n_ctx)
+        assert_o_close(o[l], O)
+        assert np.abs(lse[l].cpu().numpy() - Lr).max() <= 1e-4
+        if l in mass_layers:
+            row = mass[mass_layers.index(l)]
+            assert_rel_close(row.cpu().numpy(), M, what="mass")
+            assert abs(float(row.double().sum()) - cfg.Hq * R) <= 1e-4 * cfg.Hq * R

@@ -1,6 +1,8 @@
 """End to end: verify attention -> mass -> UV-Prune -> gather -> accept on the five
 workload configurations, GPU against oracle, with the tolerance bands for decisions that
 floating point can flip; the whole-step C-ABI entry with host buffers; two streams."""
+import ctypes as C
+
 import numpy as np
 import pytest
 import torch
@@ -342,3 +344,64 @@ def test_step_call_rejects_bad_arguments_before_queuing_anything():
     binding.verify_step(None, pp, None, device=dev, overlap=(cs, ea, eb))
     torch.cuda.current_stream().synchronize()
     assert torch.equal(kept, kept_e) and torch.equal(dk, dk_e) and torch.equal(dv, dv_e)
+
+
+def test_config2_full_step_in_the_bench_configuration():
+    """The step bench.py times, at full size: ONE pvlm_verify_step call in overlap mode over all 64 layers of
+    config 2 (head-major cache; the gather sees layer x kv_head pseudo-layers of 256-byte rows).  Selection is
+    checked against the oracle's rule on the call's own masses, every gathered byte against torch indexing, the
+    current layer's attention and the accept outcome against the oracle."""
+    cfg = wl.CONFIGS[2]
+    L, T, R, Hkv, D = cfg.n_layers, cfg.T, cfg.R, cfg.Hkv, cfg.D
+    dev = torch.device("cuda", 0)
+    g = torch.Generator(device=dev)
+    g.manual_seed(123)
+    k_base = torch.empty((L, Hkv, T, D), dtype=torch.bfloat16, device=dev)
+    v_base = torch.empty_like(k_base)
+    q = torch.empty((L, R, cfg.Hq, D), dtype=torch.bfloat16, device=dev)
+    for l in range(L):
+        k_base[l].copy_(torch.randn((Hkv, T, D), generator=g, device=dev))
+        v_base[l].copy_(torch.randn((Hkv, T, D), generator=g, device=dev))
+        q[l].copy_(torch.randn((R, cfg.Hq, D), generator=g, device=dev))
+    k, v = k_base.permute(0, 2, 1, 3), v_base.permute(0, 2, 1, 3)
+    host = {l: wl.attn_layer(cfg, l) for l in (cfg.ref_layer, cfg.cur_layer)}
+    for l, (qb, kb, vb) in host.items():
+        q[l].copy_(bf16_cuda(qb)); k[l].copy_(bf16_cuda(kb)); v[l].copy_(bf16_cuda(vb))
+    o = torch.empty_like(q)
+    lse = torch.empty((L, cfg.Hq, R), dtype=torch.float32, device=dev)
+    mass = torch.empty((2, T), dtype=torch.float32, device=dev)
+    S2 = T - cfg.m + cfg.k_keep
+    src_k, src_v = k_base.view(L * Hkv, T, 1, D), v_base.view(L * Hkv, T, 1, D)
+    dk = torch.zeros((L * Hkv, S2, 1, D), dtype=torch.bfloat16, device=dev)
+    dv = torch.zeros_like(dk)
+    kept = torch.zeros(cfg.k_keep, dtype=torch.int32, device=dev)
+    tl, dl, tok, u = wl.accept_inputs(cfg)
+    outs = dict(n_accept=torch.zeros(1, dtype=torch.int32, device=dev),
+                out_tokens=torch.zeros((1, cfg.gamma + 1), dtype=torch.int32, device=dev),
+                p_tok=torch.zeros((1, cfg.gamma), dtype=torch.float32, device=dev),
+                q_tok=torch.zeros((1, cfg.gamma), dtype=torch.float32, device=dev))
+    pa = binding.attn_params(q, k, v, cfg.n_ctx, o, lse, mass, mass_layers=[cfg.ref_layer, cfg.cur_layer])
+    pp = binding.prune_params(mass[1], mass[0], 0, cfg.m, cfg.k_keep, kept, None, src_k, src_v, dk, dv)
+    pc = binding.accept_params(*(torch.from_numpy(x).to(dev) for x in (tl, dl, tok, u)), 1.0, outs)
+    cs, ea, eb = torch.cuda.Stream(device=dev), torch.cuda.Event(), torch.cuda.Event()
+    ea.record(); eb.record()
+    torch.cuda.synchronize()
+    for _ in range(2):
+        binding.verify_step(pa, pp, pc, device=dev, overlap=(cs, ea, eb))
+    torch.cuda.current_stream().synchronize()
+    assert binding.lib().pvlm_verify_attn_check(C.byref(pa), None) == 0
+    # selection: the oracle's rule on the call's own fp32 masses, bit for bit
+    g_ref, g_cur = mass[0].cpu().numpy(), mass[1].cpu().numpy()
+    idx = select_topk(score_fp32(g_cur, g_ref, 0, cfg.m), cfg.k_keep)
+    np.testing.assert_array_equal(kept.cpu().numpy(), idx)
+    # gather: every byte of both compacted caches (torch indexing as the independent routine)
+    rows = torch.cat([torch.from_numpy(idx.astype(np.int64)).to(dev), torch.arange(cfg.m, T, device=dev)])
+    assert torch.equal(dk, src_k.index_select(1, rows)) and torch.equal(dv, src_v.index_select(1, rows))
+    # the current layer's attention and the accept outcome against the oracle
+    O, Lr, M = oracle_attn(*host[cfg.cur_layer], cfg.n_ctx)
+    assert_o_close(o[cfg.cur_layer], O)
+    assert np.abs(lse[cfg.cur_layer].cpu().numpy() - Lr).max() <= 1e-4
+    assert_rel_close(g_cur, M, what="mass")
+    r = oracle_accept(tl, dl, tok, u)
+    assert int(outs["n_accept"].item()) == r["n_accept"]
+    assert (outs["out_tokens"].cpu().numpy().ravel()[:r["n_accept"] + 1] == r["out_tokens"][:r["n_accept"] + 1]).all()
