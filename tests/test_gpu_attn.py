@@ -292,11 +292,13 @@ def test_tensor_core_and_mma_sync_paths_agree_on_random_shapes(monkeypatch):
         assert bool(((m1 - m2).abs() <= 1e-4 * m2.abs() + 1e-30).all()), tag
 
 
-def test_config2_all_64_layers_in_the_bench_launch_configuration():
-    """The launch bench.py times: all 64 layers of config 2 in ONE call (head-major cache, mass on the reference and
-    the current layer, 889 tiles and 3.5 items per persistent CTA).  Three layers hold the host-generated data of the
-    workload recipe and are checked in full against the oracle; the others are device-drawn filler of the same shape."""
-    cfg = wl.CONFIGS[2]
+@pytest.mark.parametrize("cid", [2, 3])
+def test_all_layers_in_the_bench_launch_configuration(cid):
+    """The launch bench.py times: all layers of a multi-layer config in ONE call (head-major cache, mass on the
+    reference and the current layer; config 2: 64 layers, 889 tiles and 3.5 items per persistent CTA; config 3: 80
+    layers of 88 rows per KV head).  Three layers hold the host-generated data of the workload recipe and are checked
+    in full against the oracle; the others are device-drawn filler of the same shape."""
+    cfg = wl.CONFIGS[cid]
     L, T, R = cfg.n_layers, cfg.T, cfg.R
     dev = torch.device("cuda")
     g = torch.Generator(device=dev)
