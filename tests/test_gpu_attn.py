@@ -326,3 +326,44 @@ def test_all_layers_in_the_bench_launch_configuration(cid):
             row = mass[mass_layers.index(l)]
             assert_rel_close(row.cpu().numpy(), M, what="mass")
             assert abs(float(row.double().sum()) - cfg.Hq * R) <= 1e-4 * cfg.Hq * R
+
+
+@pytest.mark.parametrize("layout", ["token", "head"])
+def test_two_million_token_context_with_layer_strides_beyond_2_31_elements(layout):
+    """Maximum-size case: 2.1 M context tokens, 8 KV heads, two layers, so that a layer of K is 2.15 G elements
+    (offsets need 64 bits) and a head-major KV head alone is 0.5 GB.  The oracle would take minutes here, so the
+    reference is the definition written with plain torch fp64 ops on the device, for two heads of the last layer
+    (the one behind the large offset); total mass must still equal heads x rows."""
+    dev = torch.device("cuda")
+    L, Hq, Hkv, D, R = 2, 16, 8, 128, 4
+    n_ctx = 2_100_000
+    T = n_ctx + R
+    g = torch.Generator(device=dev)
+    g.manual_seed(5)
+    if layout == "token":
+        k = torch.empty((L, T, Hkv, D), dtype=torch.bfloat16, device=dev)
+        v = torch.empty_like(k)
+    else:
+        kb = torch.empty((L, Hkv, T, D), dtype=torch.bfloat16, device=dev)
+        vb = torch.empty_like(kb)
+        k, v = kb.permute(0, 2, 1, 3), vb.permute(0, 2, 1, 3)
+    for l in range(L):
+        for h in range(Hkv):
+            k[l, :, h].copy_(torch.randn((T, D), generator=g, device=dev))
+            v[l, :, h].copy_(torch.randn((T, D), generator=g, device=dev))
+    q = torch.randn((L, R, Hq, D), generator=g, device=dev).to(torch.bfloat16)
+    assert k.stride(0) > 2 ** 31
+    o, lse, mass = binding.verify_attn(q, k, v, n_ctx, want_mass=True, check=True)
+    torch.cuda.synchronize()
+    for row in mass:
+        assert abs(float(row.double().sum()) - Hq * R) <= 1e-4 * Hq * R
+    l = L - 1
+    for h in (0, Hq - 1):
+        kv = h // (Hq // Hkv)
+        s = (q[l, :, h].double() @ k[l, :, kv].double().T) / np.sqrt(D)       # [R, T]
+        for r in range(R):
+            s[r, n_ctx + r + 1:] = -float("inf")
+        lse_ref = torch.logsumexp(s, dim=1)
+        o_ref = torch.exp(s - lse_ref[:, None]) @ v[l, :, kv].double()
+        assert bool(((o[l, :, h].double() - o_ref).abs() <= 1e-2 + 2e-2 * o_ref.abs()).all())
+        assert float((lse[l, h].double() - lse_ref).abs().max()) <= 1e-4
