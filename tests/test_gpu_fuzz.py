@@ -8,10 +8,11 @@ import numpy as np
 import pytest
 import torch
 
+from oracle.attention import verify_attn as oracle_attn
 from oracle.pipeline import parallel_decode as oracle_decode
 from oracle.uvprune import gather_rows, score_fp32, select_topk
 from paper_2603_19610_b200 import binding, workloads as wl
-from helpers import bits_of
+from helpers import assert_o_close, assert_rel_close, bits_of
 from test_gpu_accept import check_against_oracle
 from test_gpu_decode import gpu_decode, log_rows, make_case
 from test_gpu_prune import gpu_select
@@ -62,6 +63,15 @@ def test_attention_random_geometries(monkeypatch):
         assert bool((err <= 1e-2 + 2e-2 * o2.float().abs()).all()), tag
         assert float((l1 - l2).abs().max()) <= 1e-4, tag
         assert bool(((m1 - m2).abs() <= 1e-4 * m2.abs() + 1e-30).all()), tag
+        if L * Hq * R * T <= 2_000_000:                  # small enough for the oracle: the last layer against it as well
+            l = L - 1
+            O, Lr, M = oracle_attn(np.ascontiguousarray(bits_of(q[l])), np.ascontiguousarray(bits_of(k[l])),
+                                   np.ascontiguousarray(bits_of(v[l])), n_ctx)
+            assert_o_close(o1[l], O)
+            assert np.abs(l1[l].cpu().numpy() - Lr).max() <= 1e-4, tag
+            if ml is None or l in ml:
+                row = m1[l] if ml is None else m1[ml.index(l)]
+                assert_rel_close(row.cpu().numpy(), M, what="mass")
 
 
 def test_select_random_sizes_and_score_distributions():
