@@ -1,5 +1,6 @@
 // C-ABI entry points: host-side argument validation, workspace queries, dispatch.
 #include "pvlm_common.cuh"
+#include <cstdlib>
 
 #include <cmath>
 
@@ -10,6 +11,12 @@ static thread_local int g_last_cuda_error = 0;
 void set_cuda_error(int e) { g_last_cuda_error = e; }
 
 static thread_local cudaEvent_t g_after_main_event = nullptr;
+
+bool pdl_enabled() {
+  static const bool on = [] { const char* e = getenv("PVLM_PDL"); return !(e && e[0] == '0'); }();
+  return on;
+}
+
 void set_after_main_event(cudaEvent_t ev) { g_after_main_event = ev; }
 cudaEvent_t take_after_main_event() {
   cudaEvent_t ev = g_after_main_event;

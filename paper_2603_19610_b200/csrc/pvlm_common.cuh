@@ -15,6 +15,36 @@ constexpr float kLn2 = 0.6931471805599453f;
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
+// ---- programmatic dependent launch ------------------------------------------------------------------
+// A kernel lets the next one in the stream start its CTAs early (pdl_launch_dependents, at its top), and that one
+// blocks in pdl_wait until every kernel before it has completed and their writes are visible.  Rule for kernels
+// launched with launch_dependent(): everything read that an earlier kernel of the same call wrote, and every
+// write to memory an earlier kernel may still read, comes after pdl_wait; only work on the call's own inputs
+// (index arithmetic, barrier set-up, loads of caller-provided tensors) may precede it.  Both instructions are
+// no-ops when the launch carries no dependency.  PVLM_PDL=0 in the environment launches everything plainly.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+bool pdl_enabled();
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  if (pdl_enabled()) {
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Records a failed launch for pvlm_last_cuda_error(); returns PVLM_ERR_CUDA or PVLM_OK.
 pvlm_status check_launch();
 void set_cuda_error(int e);

@@ -35,12 +35,6 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// Programmatic dependent launch: a kernel lets the next one in the stream start its CTAs early
-// (pdl_launch_dependents), and that one blocks in pdl_wait until the kernels before it have completed and their
-// writes are visible.  Everything a kernel reads that an earlier kernel of the call wrote comes after pdl_wait.
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 constexpr int kSimRowsPerCta = 8;      // text rows per CTA of the text pass (one per warp)
 
 // Text pass, one read of the text rows from HBM: a CTA takes 8 consecutive rows; each warp computes 1 / |X_j| of
@@ -194,27 +188,15 @@ pvlm_status launch_similarity(const pvlm_similarity_params& p, cudaStream_t s) {
   a.u = (float*)(ws + align_up((size_t)parts * p.d * 4, 256));
   a.inv_norm = nullptr;
   // the second and third kernel are launched as programmatic dependents of the one before (see pdl_wait)
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr.val.programmaticStreamSerializationAllowed = 1;
-  cudaLaunchConfig_t cfg = {};
-  cfg.blockDim = dim3(256);
-  cfg.stream = s;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
   cudaError_t e = cudaSuccess;
   if (p.n > 0) sim_text_kernel<<<parts, 256, 0, s>>>(a);
-  cfg.gridDim = dim3(ceil_div(p.d, 32));
-  cfg.dynamicSmemBytes = 0;
-  e = cudaLaunchKernelEx(&cfg, sim_text_reduce_kernel, a, p.n > 0 ? parts : 0);
+  e = launch_dependent(sim_text_reduce_kernel, dim3(ceil_div(p.d, 32)), dim3(256), 0, s, a, p.n > 0 ? parts : 0);
   if (e == cudaSuccess && p.m > 0) {
     int blocks = ceil_div(p.m, 8);
     if (blocks > kNumSMs * 16) blocks = kNumSMs * 16;
     const int smem = p.d * 4;
     e = cudaFuncSetAttribute(sim_visual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    cfg.gridDim = dim3(blocks);
-    cfg.dynamicSmemBytes = smem;
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, sim_visual_kernel, a);
+    if (e == cudaSuccess) e = launch_dependent(sim_visual_kernel, dim3(blocks), dim3(256), smem, s, a);
   }
   if (e != cudaSuccess) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   return check_launch();

@@ -60,6 +60,7 @@ __device__ void accept_scan_body(const AccArgs& a, int b);
 __device__ void resid_pick_body(const AccArgs& a, int b);
 
 __global__ void __launch_bounds__(kStatThreads) row_stats_kernel(const AccArgs a) {
+  pdl_launch_dependents();
   const int chunk = blockIdx.x, row = blockIdx.y, b = blockIdx.z;
   const float* x = row_ptr(a, b, row);
   const float c = a.inv_temp * kLog2e;
@@ -185,6 +186,7 @@ __device__ __forceinline__ double warp_sum_d(double v) {
 }
 
 __global__ void __launch_bounds__(kSampThreads) resid_sums_kernel(const AccArgs a) {
+  pdl_wait();                  // the accept scan of the kernel before decides which row pair this one reads
   const int chunk = blockIdx.x, b = blockIdx.y;
   const int n = a.n_accept[b];
   const int i = chunk * kSampChunk + threadIdx.x * 4;
@@ -387,7 +389,10 @@ pvlm_status launch_spec_accept(const pvlm_accept_params& p, const AcceptPlan& pl
   const cudaError_t e = cudaMemsetAsync(a.tickets, 0, (size_t)p.batch * 2 * 4, s);
   if (e != cudaSuccess) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   row_stats_kernel<<<dim3(plan.n_stat_chunks, plan.rows, p.batch), kStatThreads, 0, s>>>(a);      // + accept scan
-  resid_sums_kernel<<<dim3(plan.n_samp_chunks, p.batch), kSampThreads, 0, s>>>(a);                // + pick
+  {
+    const cudaError_t e = launch_dependent(resid_sums_kernel, dim3(plan.n_samp_chunks, p.batch), dim3(kSampThreads), 0, s, a);   // + pick
+    if (e != cudaSuccess) set_cuda_error((int)e);
+  }
   if (p.probs_p || p.probs_q)
     write_probs_kernel<<<dim3(ceil_div(p.V, 256), plan.rows, p.batch), 256, 0, s>>>(a);
   return check_launch();

@@ -33,6 +33,7 @@ struct SelArgs {
 // Single CTA: m <= 2^24 elements, 4 radix passes of 8 bits over keys kept in
 // global/L2, then an ordered compaction.
 __global__ void __launch_bounds__(kSelThreads) uvprune_select_kernel(const SelArgs a) {
+  pdl_wait();                  // the masses may come from the kernel right before (programmatic dependent launch)
   __shared__ unsigned int hist[256];
   __shared__ unsigned int s_prefix, s_remaining;
   __shared__ int warp_eq[kSelWarps], warp_sel[kSelWarps];
@@ -143,6 +144,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& 
 // order inside a warp is (i, lane) and ordered compaction needs only ballots plus two block scans.
 template <int ITEMS>
 __global__ void __launch_bounds__(kSelThreads) uvprune_select_reg_kernel(const SelArgs a) {
+  pdl_wait();                  // the masses may come from the kernel right before (programmatic dependent launch)
   __shared__ unsigned int hist[256];
   __shared__ unsigned int hist_l[256 * 32];              // one histogram column per lane: bank = lane, so the
                                                          // atomics of a warp never collide, whatever the digits
@@ -262,6 +264,7 @@ constexpr int kSelCluster = 8;
 template <int ITEMS>
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 uvprune_select_cluster_kernel(const SelArgs a) {
+  pdl_wait();                  // the masses may come from the kernel right before (programmatic dependent launch)
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   const unsigned rank = cluster.block_rank();
@@ -436,11 +439,14 @@ pvlm_status launch_uvprune_parts(const pvlm_prune_params& p, bool select, int pa
   if (select && p.m > 0) {
     const char* impl = getenv("PVLM_SELECT_IMPL");       // "cta": single-CTA kernels only (second implementation for tests)
     const bool one_cta = impl && strcmp(impl, "cta") == 0;
-    if (!one_cta && p.m <= kSelCluster * kSelThreads * 4) uvprune_select_cluster_kernel<4><<<kSelCluster, kSelThreads, 0, s>>>(sa);
-    else if (!one_cta && p.m <= kSelCluster * kSelThreads * 16) uvprune_select_cluster_kernel<16><<<kSelCluster, kSelThreads, 0, s>>>(sa);
-    else if (!one_cta && p.m <= kSelCluster * kSelThreads * 32) uvprune_select_cluster_kernel<32><<<kSelCluster, kSelThreads, 0, s>>>(sa);
-    else if (p.m <= 32 * kSelThreads) uvprune_select_reg_kernel<32><<<1, kSelThreads, 0, s>>>(sa);
-    else uvprune_select_kernel<<<1, kSelThreads, 0, s>>>(sa);
+    const dim3 cl(kSelCluster), one(1), th(kSelThreads);
+    cudaError_t e;
+    if (!one_cta && p.m <= kSelCluster * kSelThreads * 4) e = launch_dependent(uvprune_select_cluster_kernel<4>, cl, th, 0, s, sa);
+    else if (!one_cta && p.m <= kSelCluster * kSelThreads * 16) e = launch_dependent(uvprune_select_cluster_kernel<16>, cl, th, 0, s, sa);
+    else if (!one_cta && p.m <= kSelCluster * kSelThreads * 32) e = launch_dependent(uvprune_select_cluster_kernel<32>, cl, th, 0, s, sa);
+    else if (p.m <= 32 * kSelThreads) e = launch_dependent(uvprune_select_reg_kernel<32>, one, th, 0, s, sa);
+    else e = launch_dependent(uvprune_select_kernel, one, th, 0, s, sa);
+    if (e != cudaSuccess) set_cuda_error((int)e);
   }
   if (p.src_k && part != 3) {
     GatherArgs g;

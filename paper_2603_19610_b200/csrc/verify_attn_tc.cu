@@ -241,6 +241,7 @@ __host__ __device__ constexpr int s_bufs(int nrp) { return (512 - 2 * nrp) / nrp
 template <int NRP, bool HT>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const TcArgs a) {
+  pdl_launch_dependents();                 // the merge kernel behind this one may set itself up; it waits before it reads
   constexpr int NCH = NRP / 16;            // 16-column chunks per thread
   auto CW = [](int c) constexpr { return (HT && c == NRP / 16 - 1) ? 8 : 16; };   // processed columns of chunk c
   constexpr int QBOX = NRP * 128;          // bytes of one 64-channel box of Q
@@ -801,6 +802,7 @@ __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs 
   __shared__ int s_n;
   __shared__ float s_m[4], s_l[4];
   __shared__ float4 s_acc[4][32];
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
     const long long W = a.total_tiles, C = a.n_cta;
     const long long lo = (long long)item * a.tiles_per_item, hi = lo + a.tiles_per_item;
@@ -818,6 +820,7 @@ __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs 
     s_n = n;
   }
   __syncthreads();
+  pdl_wait();                                            // the partials come from the main kernel
   const int n = s_n;
   if (n <= 8) {
     // few partials per item (long tile runs): a warp merges whole rows on its own, no block barriers
@@ -910,6 +913,7 @@ __global__ void __launch_bounds__(128) attn_tc_combine_many_kernel(const Combine
   __shared__ float s_m[4], s_l[4];
   __shared__ float4 s_acc[4][32];
   __shared__ float2 s_ml[2 * kNumSMs + 4];
+  pdl_launch_dependents();
   {
     // The CTAs whose tile ranges meet this item are consecutive: thread 0 finds the first and the last with a few
     // divisions, then one thread per CTA works out that CTA's slot (-1: a CTA without tiles, possible when there
@@ -938,6 +942,7 @@ __global__ void __launch_bounds__(128) attn_tc_combine_many_kernel(const Combine
     }
     __syncthreads();
   }
+  pdl_wait();                                            // the partials come from the main kernel
   const int n = s_n;
   const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
   auto store_row = [&](int row, float4 acc, float l, float mstar) {       // called by one warp
@@ -1027,6 +1032,7 @@ struct TcMassArgs {
 template <int NRP>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a) {
+  pdl_launch_dependents();
   constexpr int NCH = NRP / 16;
   constexpr int QBOX = NRP * 128;
   constexpr int NSB = (512 / NRP) >= 4 ? 4 : (512 / NRP);
@@ -1151,6 +1157,7 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
               *reinterpret_cast<uint4*>(sQ + (c >> 3) * QBOX + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = val[k];
             }
           }
+          pdl_wait();                                      // lse2 comes from the merge kernel (Q, K are the call's inputs)
           if (st < 128) {
             float v = 1.0e30f;
             if (st < a.rows) {
@@ -1230,6 +1237,8 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
 }
 
 __global__ void mass_reduce_tc_kernel(const float* part, float* mass, int Hkv, int T, int T_pad, long long mass_ls) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int zrow = blockIdx.y;
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= T) return;
@@ -1290,7 +1299,8 @@ template <int NRP>
 void launch_tc_mass(const CUtensorMap& mk, const TcMassArgs& a, cudaStream_t s) {
   constexpr int smem = 1024 + kMassKStages * kTileBytes + 2 * NRP * 128 + 128 * 4 + 24 * 8 + 64;
   cudaFuncSetAttribute(attn_tc_mass_kernel<NRP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  attn_tc_mass_kernel<NRP><<<a.n_cta, kThreads, smem, s>>>(mk, a);
+  const cudaError_t e = launch_dependent(attn_tc_mass_kernel<NRP>, dim3(a.n_cta), dim3(kThreads), smem, s, mk, a);
+  if (e != cudaSuccess) set_cuda_error((int)e);
 }
 
 }  // namespace
@@ -1326,7 +1336,9 @@ pvlm_status launch_attn_mass_tc(const pvlm_attn_params& p, const float* lse2, fl
     case 128: launch_tc_mass<128>(mk, a, s); break;
     default: return PVLM_ERR_UNSUPPORTED;
   }
-  mass_reduce_tc_kernel<<<dim3(ceil_div(T, 256), n_mass), 256, 0, s>>>(part_mass, p.mass, p.Hkv, T, a.T_pad, p.mass_layer_stride);
+  const cudaError_t e = launch_dependent(mass_reduce_tc_kernel, dim3(ceil_div(T, 256), n_mass), dim3(256), 0, s,
+                                         (const float*)part_mass, p.mass, p.Hkv, T, a.T_pad, p.mass_layer_stride);
+  if (e != cudaSuccess) set_cuda_error((int)e);
   return check_launch();
 }
 
@@ -1407,8 +1419,9 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
     rows_y = rows_y < 1 ? 1 : (rows_y > a.rows ? a.rows : rows_y);
     // an item's tiles are spread over at most this many CTAs, each with two partials
     const long long ctas_per_item = ((long long)plan.tiles_per_item * plan.n_cta + plan.total_tiles - 1) / plan.total_tiles + 1;
-    if (2 * ctas_per_item <= 8) attn_tc_combine_kernel<<<dim3(items, rows_y), 128, 0, s>>>(c);
-    else attn_tc_combine_many_kernel<<<dim3(items, rows_y), 128, 0, s>>>(c);
+    const cudaError_t e = 2 * ctas_per_item <= 8 ? launch_dependent(attn_tc_combine_kernel, dim3(items, rows_y), dim3(128), 0, s, c)
+                                                 : launch_dependent(attn_tc_combine_many_kernel, dim3(items, rows_y), dim3(128), 0, s, c);
+    if (e != cudaSuccess) set_cuda_error((int)e);
   }
   return check_launch();
 }
