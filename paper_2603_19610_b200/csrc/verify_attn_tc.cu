@@ -241,7 +241,6 @@ __host__ __device__ constexpr int s_bufs(int nrp) { return (512 - 2 * nrp) / nrp
 template <int NRP, bool HT>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const TcArgs a) {
-  pdl_launch_dependents();                 // the merge kernel behind this one may set itself up; it waits before it reads
   constexpr int NCH = NRP / 16;            // 16-column chunks per thread
   auto CW = [](int c) constexpr { return (HT && c == NRP / 16 - 1) ? 8 : 16; };   // processed columns of chunk c
   constexpr int QBOX = NRP * 128;          // bytes of one 64-channel box of Q
@@ -773,6 +772,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // ---- teardown (every loop above is bounded, so every thread gets here) ----
   tc_fence_before();
   __syncthreads();
+  // This CTA's work is done: the kernel behind this one may be scheduled once every CTA got here (it waits before it
+  // reads).  Not earlier: its CTAs would sit on SM slots for the whole run of this kernel and keep another stream's
+  // kernels off the SMs this launch leaves free.
+  pdl_launch_dependents();
   if (tid == 0) PHASE(7)
   if (*s_abort) {
     if (tid == 0) atomicExch(a.status, 1);
@@ -1032,7 +1035,6 @@ struct TcMassArgs {
 template <int NRP>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a) {
-  pdl_launch_dependents();
   constexpr int NCH = NRP / 16;
   constexpr int QBOX = NRP * 128;
   constexpr int NSB = (512 / NRP) >= 4 ? 4 : (512 / NRP);
@@ -1226,6 +1228,7 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
   }
   tc_fence_before();
   __syncthreads();
+  pdl_launch_dependents();                 // at the end, as in the main kernel
   if (*s_abort) {
     if (tid == 0) atomicExch(a.status, 1);
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);
