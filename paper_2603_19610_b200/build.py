@@ -1,16 +1,25 @@
-"""In-tree build of libpvlm.so (nvcc, sm_100a only)."""
+"""In-tree build of libpvlm.so (nvcc, sm_100a only).
+
+Every source is compiled to an object file of its own (in parallel, and only
+when it or a header changed), then the objects are linked into the shared
+library next to this file.
+"""
 from __future__ import annotations
 
 import os
 import shutil
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
+OBJ_DIR = os.path.join(PKG_DIR, "build")
 LIB_PATH = os.path.join(PKG_DIR, "libpvlm.so")
-SOURCES = ["pvlm_api.cu", "verify_attn.cu", "verify_attn_tc.cu", "uvprune.cu", "similarity.cu", "spec_accept.cu", "parallel_decode.cu", "acceptance_rate.cu"]
+SOURCES = ["pvlm_api.cu", "verify_attn.cu", "verify_attn_tc.cu", "uvprune.cu", "similarity.cu", "spec_accept.cu",
+           "parallel_decode.cu", "acceptance_rate.cu"]
+ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 
 def _nvcc() -> str:
@@ -20,27 +29,52 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found: libpvlm.so cannot be built")
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB_PATH):
+def _headers() -> list[str]:
+    return [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))] + \
+           [os.path.join(ROOT, "include", "pvlm.h")]
+
+
+def _stale(target: str, deps: list[str]) -> bool:
+    if not os.path.exists(target):
         return True
-    t = os.path.getmtime(LIB_PATH)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "pvlm.h")]
+    t = os.path.getmtime(target)
     return any(os.path.getmtime(d) > t for d in deps)
+
+
+def needs_build() -> bool:
+    return _stale(LIB_PATH, [os.path.join(CSRC, s) for s in SOURCES] + _headers())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB_PATH
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-           "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", LIB_PATH] + [os.path.join(CSRC, s) for s in SOURCES]
+    nvcc = _nvcc()
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    headers = _headers()
+    log: list[str] = []
+
+    def compile_one(src: str) -> str:
+        obj = os.path.join(OBJ_DIR, src[:-3] + ".o")
+        path = os.path.join(CSRC, src)
+        if force or verbose or _stale(obj, [path] + headers):
+            cmd = [nvcc, *ARCH, "-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),
+                   "-I", CSRC, "-c", path, "-o", obj]
+            if verbose:
+                cmd.insert(1, "-Xptxas=-v")
+            res = subprocess.run(cmd, capture_output=True, text=True)
+            if verbose:
+                log.append(f"==== {src}\n{res.stderr}")
+            if res.returncode != 0:
+                raise RuntimeError(f"nvcc failed on {src}:\n" + res.stdout + res.stderr)
+        return obj
+
+    with ThreadPoolExecutor(max_workers=min(len(SOURCES), os.cpu_count() or 1)) as pool:
+        objs = list(pool.map(compile_one, SOURCES))
     if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose:
-        sys.stderr.write(res.stderr)
+        sys.stderr.write("".join(log))
+    res = subprocess.run([nvcc, *ARCH, "-shared", "-o", LIB_PATH, *objs], capture_output=True, text=True)
     if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
     return LIB_PATH
 
 

@@ -29,6 +29,36 @@ def test_softmax_rows():
     np.testing.assert_allclose(softmax64(x + np.float32(1000.0)), p, rtol=1e-3)
 
 
+@pytest.mark.parametrize("temperature", [1.0, 0.5, 2.0])
+def test_lse_rows(temperature):
+    """log-sum-exp of logits / temperature, pinned four ways: scalar math.exp / math.log loops, the identity
+    lse = x_j / T - log softmax_j at the argmax and at every j, the shift law lse(x + c) = lse(x) + c / T
+    (also where exp(x) alone would overflow), and the closed form log(n) + a / T for n equal logits."""
+    from oracle.accept import lse64
+    rng = np.random.default_rng(11)
+    x = (3 * rng.standard_normal((4, 700))).astype(np.float32)
+    got = lse64(x, temperature)
+    assert got.shape == (4,) and got.dtype == np.float64
+    want = np.array([math.log(sum(math.exp(float(v) / temperature) for v in row)) for row in x])
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    p = softmax64(x, temperature)
+    j = p.argmax(axis=1)
+    np.testing.assert_allclose(got, x[np.arange(4), j].astype(np.float64) / temperature - np.log(p[np.arange(4), j]), atol=1e-12)
+    np.testing.assert_allclose(got[:, None] - x.astype(np.float64) / temperature, -np.log(p), atol=1e-9)
+    np.testing.assert_allclose(lse64(x + np.float32(900.0), temperature),
+                               lse64((x + np.float32(900.0)).astype(np.float64) - 900.0, temperature) + 900.0 / temperature, atol=1e-9)
+    np.testing.assert_allclose(lse64(np.full((2, 37), 1.25, np.float32), temperature), math.log(37) + 1.25 / temperature, atol=1e-13)
+    # a masked entry (-inf) adds nothing; a single entry is its own lse
+    y = x.copy()
+    y[:, 5] = -np.inf
+    np.testing.assert_allclose(lse64(y, temperature), lse64(np.delete(x, 5, axis=1), temperature), atol=1e-12)
+    np.testing.assert_allclose(lse64(x[:, :1], temperature), x[:, 0].astype(np.float64) / temperature, atol=1e-13)
+    # the values spec_accept reports are these
+    r = spec_accept(x, x[:3] + np.float32(0.5), [0, 1, 2], np.full(4, 0.5, np.float32), temperature)
+    np.testing.assert_array_equal(r["lse_p"], got)
+    np.testing.assert_allclose(r["lse_q"], got[:3] + 0.5 / temperature, atol=1e-6)
+
+
 def test_inverse_cdf_rule():
     w = np.array([0.0, 0.2, 0.0, 0.3, 0.5, 0.0])
     assert inverse_cdf(w, 0.0) == 1            # zero-weight token 0 is never chosen
