@@ -56,6 +56,23 @@ int pvlm_last_cuda_error(void);
 /* Library version: major * 1000 + minor. */
 int pvlm_version(void);
 
+/* Process-wide switches for tests and A/B measurements; none selects a CPU path and none is needed for
+ * normal use.  Their defaults are read ONCE from the environment (the variable named beside each), so the
+ * launch path of every call is free of environment lookups; afterwards only this function changes them.
+ * It returns the previous value, or -1 for an unknown option or a negative value.  A change takes effect
+ * for calls (and workspace queries) issued after it returns; do not change a switch between a workspace
+ * query and the call it sizes. */
+enum {
+  PVLM_OPT_ATTN_MMA_SYNC = 0,  /* 1: pvlm_verify_attn runs its first implementation (mma.sync kernels) instead of
+                                  the tcgen05 one: a second implementation for tests.  PVLM_ATTN_IMPL=mma      */
+  PVLM_OPT_SELECT_ONE_CTA = 1, /* 1: the Top-K selection runs its single-CTA kernels instead of the 8-CTA cluster
+                                  kernel: a second implementation for tests.  PVLM_SELECT_IMPL=cta             */
+  PVLM_OPT_ATTN_MAX_CTAS = 2,  /* n > 0: the tcgen05 attention uses at most n persistent CTAs, so that small test
+                                  shapes exercise long tile runs and many segments per CTA.  PVLM_TC_CTAS=n    */
+  PVLM_OPT_COUNT = 3
+};
+int pvlm_set_option(int option, int value);
+
 /* ------------------------------------------------------------------------
  * Window-verify grouped-query attention with attention-mass emission.
  *
@@ -210,6 +227,11 @@ pvlm_status pvlm_uvprune_similarity(const pvlm_similarity_params *p, void *strea
  * Supported: 0 <= gamma <= 64; 1 <= V < 2^31; 1 <= batch <= 65535.  Rows are
  * read with 16-byte loads when the logit base pointers are 16-byte aligned
  * and all logit strides are multiples of 4 elements, else element by element.
+ *
+ * One kernel launch.  Inside it a few thread blocks wait (for microseconds)
+ * for the block that determines n_accept; that wait is bounded to one second,
+ * and if it ever expired the drawn token would be missing:
+ * out_tokens[n_accept] == -1 is the mark of that failure.
  * ---------------------------------------------------------------------- */
 typedef struct {
   const float *target_logits;  /* fp32 [batch][gamma+1][V]                                    */
@@ -231,6 +253,36 @@ typedef struct {
 
 size_t pvlm_spec_accept_workspace_bytes(const pvlm_accept_params *p);
 pvlm_status pvlm_spec_accept(const pvlm_accept_params *p, void *stream);
+
+/* ------------------------------------------------------------------------
+ * The two decisions of the step on their own, from given scores / probabilities.
+ *
+ * Kept indices and accepted lengths are integer results of floating-point
+ * inputs.  These two calls take those inputs from the caller instead of
+ * computing them, so that a test can feed values computed elsewhere (e.g. by an
+ * independent CPU implementation) and compare the integer results bit for bit.
+ * They run the same device code as the full calls.
+ *
+ * pvlm_select_from_scores: Top-K of paper Eq. 3 over given scores.
+ *   score fp32 [m] (device); kept_idx int32 [k] out, ascending; the k largest
+ *   scores, equal scores lower index first, -0.0 == +0.0, NaN below every
+ *   number: pvlm_uvprune_select_gather with mass_cur = score, mass_ref = NULL,
+ *   vis_start = 0 and no gather.  Workspace as pvlm_uvprune_workspace_bytes
+ *   reports for the same m.  Errors as for that call.
+ *
+ * pvlm_accept_from_probs: the accept rule of paper Sec. 2.2 over given token
+ *   probabilities.  p_tok, q_tok fp32 [batch][gamma] (device): p_t(x_t) and
+ *   q_t(x_t) of the drafted tokens; uniforms fp32 [batch][uniform_stride]
+ *   (device), the first gamma of each row used (uniform_stride >= gamma; pass
+ *   gamma + 1 for the array pvlm_spec_accept takes); n_accept int32 [batch]
+ *   out: the first t with not (u_t * q_t < p_t), evaluated as in
+ *   pvlm_spec_accept (one rounded fp32 multiply, strict compare), or gamma if
+ *   there is none.  0 <= gamma, 1 <= batch.  No workspace.
+ * ---------------------------------------------------------------------- */
+pvlm_status pvlm_select_from_scores(const float *score, int m, int k, int *kept_idx, void *workspace,
+                                    size_t workspace_bytes, void *stream);
+pvlm_status pvlm_accept_from_probs(const float *p_tok, const float *q_tok, const float *uniforms, int uniform_stride,
+                                   int gamma, int batch, int *n_accept, void *stream);
 
 /* ------------------------------------------------------------------------
  * One whole verify -> prune -> accept step from HOST-side step inputs.

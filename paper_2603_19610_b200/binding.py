@@ -106,7 +106,8 @@ EXPORTS = ("pvlm_status_string", "pvlm_last_cuda_error", "pvlm_version",
            "pvlm_spec_accept_workspace_bytes", "pvlm_spec_accept", "pvlm_verify_step",
            "pvlm_uvprune_select_static", "pvlm_uvprune_similarity_workspace_bytes", "pvlm_uvprune_similarity", "pvlm_window_size",
            "pvlm_parallel_decode_workspace_bytes", "pvlm_parallel_decode",
-           "pvlm_acceptance_rate_workspace_bytes", "pvlm_acceptance_rate")
+           "pvlm_acceptance_rate_workspace_bytes", "pvlm_acceptance_rate",
+           "pvlm_select_from_scores", "pvlm_accept_from_probs", "pvlm_set_option")
 
 
 def lib() -> C.CDLL:
@@ -145,6 +146,13 @@ def lib() -> C.CDLL:
             L.pvlm_uvprune_select_static.restype = C.c_int
             L.pvlm_uvprune_select_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                                      C.c_void_p, C.c_void_p, C.c_void_p]
+            L.pvlm_set_option.restype = C.c_int
+            L.pvlm_set_option.argtypes = [C.c_int, C.c_int]
+            L.pvlm_select_from_scores.restype = C.c_int
+            L.pvlm_select_from_scores.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+            L.pvlm_accept_from_probs.restype = C.c_int
+            L.pvlm_accept_from_probs.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                                 C.c_void_p]
             _LIB = L
     return _LIB
 
@@ -160,6 +168,17 @@ def _workspace(dev: torch.device, key: str, nbytes: int) -> torch.Tensor:
         buf = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=dev)
         _WS[k] = buf
     return buf
+
+
+OPTIONS = {"attn_mma_sync": 0, "select_one_cta": 1, "attn_max_ctas": 2}
+
+
+def set_option(name: str, value: int) -> int:
+    """Process-wide test / A-B switch (see pvlm_set_option).  Returns the previous value."""
+    prev = lib().pvlm_set_option(OPTIONS[name], int(value))
+    if prev < 0:
+        raise ValueError(f"pvlm_set_option({name}, {value}) refused")
+    return prev
 
 
 def _ptr(t):
@@ -384,6 +403,40 @@ def uvprune_select_static(mass_cur, mass_ref, vis_start: int, m: int, k: int, ke
     if st != 0:
         raise PvlmError(st, "pvlm_uvprune_select_static")
     return kept_idx
+
+
+def select_from_scores(score, k: int, *, workspace=None):
+    """Top-K over given fp32 scores (see pvlm_select_from_scores).  Returns kept_idx int32 [k], ascending."""
+    _need_cuda(score)
+    assert score.dtype == torch.float32 and score.dim() == 1 and score.is_contiguous()
+    dev, m = score.device, score.numel()
+    kept = torch.empty(k, dtype=torch.int32, device=dev)
+    pp = PruneParams()
+    pp.m = m
+    need = lib().pvlm_uvprune_workspace_bytes(C.byref(pp))
+    ws = workspace if workspace is not None else _workspace(dev, "prune", need)
+    st = lib().pvlm_select_from_scores(_ptr(score), m, k, _ptr(kept), _ptr(ws), ws.numel(), _stream(dev))
+    if st != 0:
+        raise PvlmError(st, "pvlm_select_from_scores")
+    return kept
+
+
+def accept_from_probs(p_tok, q_tok, uniforms):
+    """First rejection from given token probabilities (see pvlm_accept_from_probs).
+    p_tok, q_tok fp32 [batch, gamma] (or [gamma]); uniforms fp32 [batch, >= gamma].  Returns n_accept int32 [batch]."""
+    _need_cuda(p_tok, q_tok, uniforms)
+    if p_tok.dim() == 1:
+        p_tok, q_tok, uniforms = p_tok[None], q_tok[None], uniforms[None]
+    B, gamma = p_tok.shape
+    assert q_tok.shape == (B, gamma) and uniforms.shape[0] == B and uniforms.shape[1] >= gamma
+    assert p_tok.dtype == q_tok.dtype == uniforms.dtype == torch.float32
+    assert p_tok.is_contiguous() and q_tok.is_contiguous() and uniforms.stride(1) == 1
+    n = torch.empty(B, dtype=torch.int32, device=p_tok.device)
+    st = lib().pvlm_accept_from_probs(_ptr(p_tok), _ptr(q_tok), _ptr(uniforms), uniforms.stride(0) if B > 1 else uniforms.shape[1],
+                                      gamma, B, _ptr(n), _stream(p_tok.device))
+    if st != 0:
+        raise PvlmError(st, "pvlm_accept_from_probs")
+    return n
 
 
 def uvprune_similarity(hidden, vis_start: int, m: int, text_start: int, n: int, *, out=None, workspace=None):

@@ -2,7 +2,9 @@
 #include "pvlm_common.cuh"
 #include <cstdlib>
 
+#include <atomic>
 #include <cmath>
+#include <cstring>
 
 namespace pvlm {
 
@@ -16,6 +18,25 @@ bool pdl_enabled() {
   static const bool on = [] { const char* e = getenv("PVLM_PDL"); return !(e && e[0] == '0'); }();
   return on;
 }
+
+// Process-wide switches.  Their defaults come from the environment, read once when the first one is looked at;
+// after that only pvlm_set_option changes them, so no call reads the environment on its launch path.
+static std::atomic<int>* option_slots() {
+  static std::atomic<int> slots[PVLM_OPT_COUNT];
+  static const bool init = [] {
+    const char* e = getenv("PVLM_ATTN_IMPL");
+    slots[PVLM_OPT_ATTN_MMA_SYNC].store(e && strcmp(e, "mma") == 0);
+    e = getenv("PVLM_SELECT_IMPL");
+    slots[PVLM_OPT_SELECT_ONE_CTA].store(e && strcmp(e, "cta") == 0);
+    e = getenv("PVLM_TC_CTAS");
+    slots[PVLM_OPT_ATTN_MAX_CTAS].store(e ? atoi(e) : 0);
+    return true;
+  }();
+  (void)init;
+  return slots;
+}
+
+int option_value(int option) { return option_slots()[option].load(std::memory_order_relaxed); }
 
 void set_after_main_event(cudaEvent_t ev) { g_after_main_event = ev; }
 cudaEvent_t take_after_main_event() {
@@ -62,7 +83,13 @@ const char* pvlm_status_string(pvlm_status s) {
 
 int pvlm_last_cuda_error(void) { return g_last_cuda_error; }
 
-int pvlm_version(void) { return 1000; }
+int pvlm_version(void) { return 1001; }
+
+int pvlm_set_option(int option, int value) {
+  if (option < 0 || option >= PVLM_OPT_COUNT) return -1;
+  if (value < 0) return -1;
+  return option_slots()[option].exchange(value);
+}
 
 size_t pvlm_verify_attn_workspace_bytes(const pvlm_attn_params* p) {
   AttnPlan plan;
@@ -205,6 +232,25 @@ pvlm_status pvlm_spec_accept(const pvlm_accept_params* p, void* stream) {
   const pvlm_status v = validate_accept(p, plan);
   if (v != PVLM_OK) return v;
   return launch_spec_accept(*p, plan, (cudaStream_t)stream);
+}
+
+pvlm_status pvlm_select_from_scores(const float* score, int m, int k, int* kept_idx, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+  pvlm_prune_params p = {};
+  p.mass_cur = score;
+  p.m = m;
+  p.k = k;
+  p.kept_idx = kept_idx;
+  p.workspace = workspace;
+  p.workspace_bytes = workspace_bytes;
+  return pvlm_uvprune_select_gather(&p, stream);
+}
+
+pvlm_status pvlm_accept_from_probs(const float* p_tok, const float* q_tok, const float* uniforms, int uniform_stride,
+                                   int gamma, int batch, int* n_accept, void* stream) {
+  if (gamma < 0 || batch < 1 || uniform_stride < gamma || !n_accept) return PVLM_ERR_INVALID_ARG;
+  if (gamma > 0 && (!p_tok || !q_tok || !uniforms)) return PVLM_ERR_INVALID_ARG;
+  return launch_accept_from_probs(p_tok, q_tok, uniforms, uniform_stride, gamma, batch, n_accept, (cudaStream_t)stream);
 }
 
 pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {

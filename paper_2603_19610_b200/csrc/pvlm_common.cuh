@@ -27,6 +27,8 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 bool pdl_enabled();
+// Current value of a process-wide switch (pvlm_set_option; the default comes from the environment, read once).
+int option_value(int option);
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
@@ -98,11 +100,15 @@ pvlm_status launch_similarity(const pvlm_similarity_params& p, cudaStream_t s);
 // ---- accept -----------------------------------------------------------------
 struct AcceptPlan {
   int rows;             // 2 * gamma + 1 logit rows per sequence
-  int stat_chunk, n_stat_chunks;      // row-statistics chunking over V
-  int samp_chunk, n_samp_chunks;      // resampling chunking over V
-  size_t off_stats, off_lse, off_n, off_csum, off_clast, total;
+  int n_stat_chunks;    // statistics CTAs per row
+  int stat_chunk;       // elements per statistics CTA
+  int team;             // CTAs of the tail team per sequence (cluster size)
+  int nit;              // residual-pass iterations per warp of the team
+  size_t off_stats, off_lse, off_sync, total;
 };
 bool make_accept_plan(const pvlm_accept_params& p, AcceptPlan& plan);
 pvlm_status launch_spec_accept(const pvlm_accept_params& p, const AcceptPlan& plan, cudaStream_t s);
+pvlm_status launch_accept_from_probs(const float* p_tok, const float* q_tok, const float* uniforms, long long u_stride,
+                                     int gamma, int batch, int* n_accept, cudaStream_t s);
 
 }  // namespace pvlm

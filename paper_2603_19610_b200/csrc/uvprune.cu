@@ -3,8 +3,6 @@
 // compacted draft cache.
 #include "pvlm_common.cuh"
 #include <cooperative_groups.h>
-#include <cstdlib>
-#include <cstring>
 #include <mutex>
 
 namespace pvlm {
@@ -166,9 +164,6 @@ __global__ void __launch_bounds__(kSelThreads) uvprune_select_reg_kernel(const S
     }
   }
   if (a.k == 0) return;
-#ifdef PVLM_SEL_PROFILE
-  long long pt[6]; pt[0] = clock64();
-#endif
   if (tid == 0) { s_prefix = 0u; s_remaining = (unsigned)a.k; }
   uint32_t mask = 0u;
   for (int shift = 24; shift >= 0; shift -= 8) {
@@ -214,9 +209,6 @@ __global__ void __launch_bounds__(kSelThreads) uvprune_select_reg_kernel(const S
   const uint32_t tau = s_prefix;
   const int take_eq = (int)s_remaining;
   const unsigned lt_mask = (1u << lane) - 1u;
-#ifdef PVLM_SEL_PROFILE
-  pt[1] = clock64();
-#endif
   // equals per warp -> rank of every equal element in index order
   int warp_eq = 0;
 #pragma unroll
@@ -246,11 +238,6 @@ __global__ void __launch_bounds__(kSelThreads) uvprune_select_reg_kernel(const S
     if ((selbits >> i) & 1u) a.kept[pos + __popc(sel_b & lt_mask)] = base + i * 32;
     pos += __popc(sel_b);
   }
-#ifdef PVLM_SEL_PROFILE
-  pt[2] = clock64();
-  __syncthreads();
-  if (tid == 0) { a.kept[0] = (int)(pt[1] - pt[0]); a.kept[1] = (int)(pt[2] - pt[1]); a.kept[2] = (int)(pt[0] & 0x7fffffff); }
-#endif
 }
 
 // Cluster variant: 8 CTAs (one thread-block cluster, 8 SMs) share the selection.  CTA r owns the
@@ -437,8 +424,7 @@ pvlm_status launch_uvprune_parts(const pvlm_prune_params& p, bool select, int pa
   sa.m = p.m;
   sa.k = p.k;
   if (select && p.m > 0) {
-    const char* impl = getenv("PVLM_SELECT_IMPL");       // "cta": single-CTA kernels only (second implementation for tests)
-    const bool one_cta = impl && strcmp(impl, "cta") == 0;
+    const bool one_cta = option_value(PVLM_OPT_SELECT_ONE_CTA) != 0;    // single-CTA kernels only: the tests' second implementation
     const dim3 cl(kSelCluster), one(1), th(kSelThreads);
     cudaError_t e;
     if (!one_cta && p.m <= kSelCluster * kSelThreads * 4) e = launch_dependent(uvprune_select_cluster_kernel<4>, cl, th, 0, s, sa);
@@ -471,11 +457,7 @@ pvlm_status launch_uvprune_parts(const pvlm_prune_params& p, bool select, int pa
       long long blocks = (total + 255) / 256;
       // Short-lived CTAs (four K + V copies per thread) measured faster than a resident grid that loops (419 vs 440 µs on
       // the 64-layer gather), and they give SM slots back quickly when the launch runs beside another stream's kernels.
-      long long cap = (blocks + 3) / 4;
-      if (const char* e = getenv("PVLM_GATHER_ITERS")) {           // tuning hook: copies per thread (0 = resident grid)
-        const int it = atoi(e);
-        cap = it <= 0 ? (long long)kNumSMs * 16 : (blocks + it - 1) / it;
-      }
+      const long long cap = (blocks + 3) / 4;
       if (blocks > cap) blocks = cap;
       uvprune_gather_kernel<<<(int)blocks, 256, 0, s>>>(g);
     }

@@ -408,12 +408,13 @@ bool make_attn_plan(const pvlm_attn_params& p, AttnPlan& plan) {
   off += align_up((size_t)p.n_layers * p.Hq * p.R * 4, 256);
   plan.off_part_mass = off;
   if (p.mass) {
+    if (p.mass_layers && (p.n_mass_layers < 1 || p.n_mass_layers > 8)) return false;
     const int n_mass = p.mass_layers ? p.n_mass_layers : p.n_layers;
     off += align_up((size_t)n_mass * p.Hkv * align_up(plan.T, kAttnBN) * 4, 256);
   }
   // main pass on the tcgen05 kernel whenever it applies (PVLM_ATTN_IMPL=mma forces the mma.sync kernel)
-  const char* impl = getenv("PVLM_ATTN_IMPL");
-  plan.use_tc = (p.D == 128 || p.D == 64) && !(impl && strcmp(impl, "mma") == 0) && make_attn_tc_plan(p, plan.tc);
+  const bool force_mma = option_value(PVLM_OPT_ATTN_MMA_SYNC) != 0;
+  plan.use_tc = (p.D == 128 || p.D == 64) && !force_mma && make_attn_tc_plan(p, plan.tc);
   plan.off_tc = off;
   if (plan.use_tc) off += align_up(plan.tc.total, 256);
   plan.total = off;

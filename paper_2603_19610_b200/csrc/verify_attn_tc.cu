@@ -10,13 +10,16 @@
 //
 // Inside a CTA (12 warps = 3 warpgroups; registers are moved from warpgroup 0 to the softmax
 // warpgroups with setmaxnreg):
-//   warp 0       TMA producer: K and V tiles (two 64-channel boxes each, 128-byte swizzle) into
-//                separate 2-deep shared-memory rings, completion on mbarriers.
-//   warp 1       MMA issuer (one thread): S^T = K . Q^T  (M = 128 keys, N = padded query rows,
-//                K = 128 channels) into one of up to four TMEM score buffers, then O^T += V^T . P^T
-//                (M = 128 channels, N = rows, K = 128 keys) into a TMEM output accumulator.  (Two
-//                separate issuer threads were tried: they let the two softmax groups fall into step,
-//                which loses the overlap between them.)
+//   warp 0       TMA producer (one lane): K and V tiles (two 64-channel boxes each, 128-byte swizzle)
+//                into ONE shared ring of 3 to 5 slots of 32 KB, in the order the issuer consumes them
+//                (K(0..lookahead), V(0), K(lookahead+1), V(1), ...); completion on mbarriers.
+//   warp 1       MMA issuer: the whole warp walks the tile loop converged (counters, barrier
+//                addresses and descriptors are warp-uniform) and one elected lane issues
+//                S^T = K . Q^T  (M = 128 keys, N = padded query rows, K = 128 channels) into one of up
+//                to four TMEM score buffers, then O^T += V^T . P^T  (M = 128 channels, N = rows,
+//                K = 128 keys) into a TMEM output accumulator, and commits the barriers that free
+//                the ring slots.  (Two separate issuer threads were tried: they let the two softmax
+//                groups fall into step, which loses the overlap between them.)
 //   warps 4..11  two softmax groups working on alternate tiles, each with its own accumulator,
 //                reference and row sums (two interleaved online-softmax streams).  A thread owns
 //                one key (TMEM lane) of its group's tile and all query-row columns, so exp2, the
@@ -33,7 +36,6 @@
 
 #include <cuda.h>
 
-#include <cstdlib>
 
 namespace pvlm {
 
@@ -205,30 +207,6 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
          (1ull << 46) | ((uint64_t)layout << 61);
 }
 
-#ifdef PVLM_TC_PROFILE
-#define PROF_DECL long long prof_t0 = 0; long long prof_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-#define PROF_START prof_t0 = clock64();
-#define PROF_ADD(i) { const long long now = clock64(); prof_acc[i] += now - prof_t0; prof_t0 = now; }
-#define PROF_DUMP(base) { for (int pi = 0; pi < 12; ++pi) a.status[(base) + pi] = (int)(prof_acc[pi] >> 4); }
-// event trace of tiles 400..407 of CTA 0: status[64 + ev * 8 + (tile - 400)] = clock
-#define TRACE_T0(ev, j) { if (t == 0) TRACE(ev, j) }
-#define TRACE(ev, j) { if (blockIdx.x == 0 && (j) >= 400u && (j) < 408u) a.status[64 + (ev) * 8 + ((j) - 400u)] = (int)(clock64() & 0x7fffffff); }
-#else
-#define PROF_DECL
-#define PROF_START
-#define PROF_ADD(i)
-#define PROF_DUMP(base) {}
-#define TRACE(ev, j)
-#define TRACE_T0(ev, j)
-#endif
-// phase marks of CTA 0 (first time each is reached): status[200 + i] = clock.  Also available without the per-tile
-// counters above (PVLM_TC_PHASES), which disturb a short run.
-#if defined(PVLM_TC_PROFILE) || defined(PVLM_TC_PHASES)
-#define PHASE(i) { if (blockIdx.x == 0 && a.status[200 + (i)] == 0) a.status[200 + (i)] = (int)(clock64() & 0x7fffffff); }
-#else
-#define PHASE(i) {}
-#endif
-
 // ---------------------------------------------------------------------------------------------
 // The kernel.  NRP = query rows per KV head padded to a multiple of 16 (MMA N), NRP <= 96.
 // ---------------------------------------------------------------------------------------------
@@ -274,7 +252,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   auto bar = [&](int i) { return smem_addr(bars + i); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (tid == 0) PHASE(0)
 
   // ---- this CTA's range of the flattened tile sequence ----
   const long long W = a.total_tiles;
@@ -305,7 +282,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
-  if (tid == 0) PHASE(1)
   const uint32_t tmem_O = tmem;                    // O accumulators of the two softmax groups: columns [g*NRP, (g+1)*NRP)
   const uint32_t tmem_S = tmem + 2 * NRP;          // score buffers
 
@@ -317,24 +293,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // per segment K(0..lookahead), V(0), K(lookahead+1), V(1), ...  It runs ahead across segment
       // boundaries as far as free slots allow.
       if (lane == 0) {
-        PROF_DECL
         uint32_t u = 0;                          // loads issued so far (ring position)
         uint32_t jt = 0;
         bool ok = true;
         auto load = [&](const CUtensorMap* map, uint32_t full_bar, long long f) -> bool {
           const uint32_t slot = u % NS;
-          PROF_START
           if (u >= NS && !mbar_wait(bar(EMPTY + slot), ((u / NS) - 1) & 1, s_abort)) return false;
-          PROF_ADD(0)
           const int item = (int)(f / Tt), tile = (int)(f - (long long)item * Tt);
           const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
           const uint32_t dst = smem_addr(sRing + slot * kTileBytes);
-          PHASE(8)
           mbar_expect_tx(full_bar, kTileBytes);
           tma_load_4d(dst, map, full_bar, 0, kvh, tile * kTile, layer);
           tma_load_4d(dst + kBoxBytes, map, full_bar, 64, kvh, tile * kTile, layer);
           ++u;
-          PROF_ADD(2)
           return true;
         };
         for (long long f = f_begin; f < f_end && ok;) {
@@ -352,7 +323,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           jt += n;
           f = seg_end;
         }
-        if (blockIdx.x == 0) PROF_DUMP(4)
       }
     } else if (warp == 1) {
       // =========================== MMA issuer ===========================
@@ -367,32 +337,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const uint64_t desc_v0 = make_desc(smem_addr(sRing), kBoxBytes, 1024, 2), desc_p0 = make_desc(smem_addr(sP), 128, 2048, 0);
         uint32_t u = 0;            // ring position (same sequence as the producer's)
         bool ok = true;
-        PROF_DECL
         uint32_t jt = 0;           // tiles issued by this CTA so far (ring phases run across segments)
         int seg = 0;
-#ifdef PVLM_TC_PROFILE
-        if (blockIdx.x == 0) {     // micro-timings of the synchronisation primitives (cycles per operation)
-          mbar_wait(bar(Q_READY), 0, s_abort);
-          long long c0 = clock64();
-          for (int r = 0; r < 64; ++r) mbar_wait(bar(Q_READY), 0, s_abort);
-          long long c1 = clock64();
-          for (int r = 0; r < 64; ++r) tc_fence_after();
-          long long c2 = clock64();
-          a.status[140] = (int)((c1 - c0) / 64);
-          a.status[141] = (int)((c2 - c1) / 64);
-        }
-#endif
         auto wait_all = [&](uint32_t b, uint32_t parity) -> bool {     // a vote makes the outcome provably warp-uniform
           return __all_sync(0xffffffffu, mbar_wait(b, parity, s_abort));
         };
         auto issue_qk = [&](uint32_t j) -> bool {
           const uint32_t slot = u % NS, sb = j % NSB;
           ++u;
-          PROF_START
           if (!wait_all(bar(K_FULL + (j & 3)), (j >> 2) & 1)) return false;
-          if (lane == 0) PHASE(10)
-          PROF_ADD(0)
-          TRACE(0, j)
           tc_fence_after();
           const uint64_t dk = desc_k0 + (uint64_t)((slot * kTileBytes) >> 4);
           const uint32_t d_tmem = tmem_S + sb * NRP;
@@ -406,9 +359,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             tc_commit(bar(EMPTY + slot));
           }
           __syncwarp();
-          if (lane == 0) PHASE(11)
-          PROF_ADD(2)
-          TRACE(1, j)
           return true;
         };
         for (long long f = f_begin; f < f_end && ok; ++seg) {
@@ -416,7 +366,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
           const int n = (int)(seg_end - f);
           if (!wait_all(bar(Q_READY), seg & 1)) { ok = false; break; }
-          if (lane == 0) PHASE(9)
           tc_fence_after();
           int issued = 0;                                  // score tiles of this segment already issued
           for (int i = 0; i < n; ++i) {
@@ -428,12 +377,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             if (!ok) break;
             const uint32_t slot = u % NS, g = j & 1;
             ++u;
-            PROF_START
             if (i == 0 && seg > 0 && !wait_all(bar(O_FREE), (seg - 1) & 1)) { ok = false; break; }
-            PROF_ADD(3)
             if (!wait_all(bar(P_FULL + (j & 3)), (j >> 2) & 1)) { ok = false; break; }     // P stored and V landed
-            PROF_ADD(5)
-            TRACE(2, j)
             tc_fence_after();
             const uint64_t dv = desc_v0 + (uint64_t)((slot * kTileBytes) >> 4), dp = desc_p0 + (uint64_t)((g * PBYTES) >> 4);
             const uint32_t d_tmem = tmem_O + g * NRP;
@@ -446,8 +391,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               tc_commit(bar(EMPTY + slot));
             }
             __syncwarp();
-            PROF_ADD(6)
-            TRACE(3, j)
           }
           if (!ok) break;
           if (elect_one()) tc_commit(bar(O_FULL));
@@ -455,7 +398,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           jt += n;
           f = seg_end;
         }
-        if (blockIdx.x == 0 && lane == 0) PROF_DUMP(16)
       }
     } else if (warp >= 4) {
       // =========================== softmax warps ===========================
@@ -478,7 +420,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       uint32_t jt = 0;
       int seg = 0;
       bool ok = true;
-      PROF_DECL
       auto group_sync = [&]() { asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory"); };
       auto group_or = [&](bool pred) -> bool {
         uint32_t out;
@@ -526,7 +467,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       };
       q_load((int)(f_begin / Tt));
       q_store();
-      if (st == 0) PHASE(2)
       for (long long f = f_begin; f < f_end; ++seg) {
         const int item = (int)(f / Tt), tile0 = (int)(f - (long long)item * Tt);
         const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
@@ -546,11 +486,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const uint32_t s_addr = tmem_S + lane_addr + sb * NRP;
           // A failed wait never leaves this loop on its own (the rest of the group would be left at a
           // named barrier): it clears `ok`, and the vote below takes all 128 threads out together.
-          PROF_START
           ok &= mbar_wait(bar(S_FULL + sb), (j / NSB) & 1, s_abort);
-          PROF_ADD(0)
-          if (st == 0) PHASE(3)
-          TRACE_T0(4, j)
           tc_fence_after();
           if (i == i_first) {
             // First tile of this group's stream: instead of going through the reference-replacement path (row
@@ -585,7 +521,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             for (int c = 0; c < NCH; ++c)
               if (CW(c) == 16) tmem_ld16(s_addr + c * 16, xr[c]); else tmem_ld8_lo(s_addr + c * 16, xr[c]);
             tmem_wait_ld();
-            PROF_ADD(8)
             float xm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
             const float4* m4 = reinterpret_cast<const float4*>(m_s);
 #pragma unroll
@@ -635,11 +570,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           for (int attempt = 0; attempt < 2; ++attempt) {
             load_x();
             if (attempt == 1) break;
-            PROF_ADD(1)
-            TRACE_T0(5, j)
             const bool slow = group_or((xmax > kRescaleThreshold) || !ok);
-            PROF_ADD(2)
-            TRACE_T0(6, j)
             if (!slow) break;
             if (group_or(!ok)) { aborted = true; break; }              // uniform across the group
             // ------- slow path: new per-row reference, rescale row sums and the accumulator -------
@@ -687,11 +618,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             }
           }
           if (aborted) break;
-          PROF_ADD(3)
           // ---- probabilities, running sums, bf16 P in the MN-major core-matrix layout ----
           if (i >= 2) ok &= mbar_wait(bar(P_FREE + g), ((j >> 1) - 1) & 1, s_abort);
-          PROF_ADD(4)
-          TRACE_T0(7, j)
           unsigned char* pdst = sP + g * PBYTES + t * 16;
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
@@ -709,16 +637,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                     make_uint4(pack2(p[8], p[9]), pack2(p[10], p[11]), pack2(p[12], p[13]), pack2(p[14], p[15]));
             }
           }
-          PROF_ADD(5)
           fence_proxy_async();
           tc_fence_before();                    // the score buffer has been read: this arrival also releases it
           mbar_arrive(bar(P_FULL + (j & 3)));
-          if (st == 0) PHASE(4)
-          PROF_ADD(6)
-          TRACE_T0(8, j)
         }
         // both groups leave together: the exit vote is per group, so agree across groups here
-        if (st == 0) PHASE(5)
         if (softmax_bar_or(aborted)) break;
         // Both groups have read the scores of their last tiles, so every score MMA of this segment is done and Q is
         // free: the next item's Q goes in now, and the issuer starts that segment's score MMAs while the epilogue
@@ -759,13 +682,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           a.part_ml[(slot * NRP + t) * 2 + 1] = has_tiles ? l : 0.f;
         }
         group_sync();
-        if (st == 0) PHASE(6)
-        PROF_ADD(7)
         jt += n;
         f = seg_end;
       }
-      if (blockIdx.x == 0 && st == 0) PROF_DUMP(28)
-      if (blockIdx.x == 0 && st == 255) PROF_DUMP(40)
     }
   }
 
@@ -776,7 +695,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // reads).  Not earlier: its CTAs would sit on SM slots for the whole run of this kernel and keep another stream's
   // kernels off the SMs this launch leaves free.
   pdl_launch_dependents();
-  if (tid == 0) PHASE(7)
   if (*s_abort) {
     if (tid == 0) atomicExch(a.status, 1);
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);     // let copies / MMAs in flight land before TMEM is released
@@ -1254,17 +1172,17 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Looked up once per process; the initialisation of a function-local static is thread-safe, so host threads
+// that make their first attention call at the same time all see the finished pointer.
 EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  static const EncodeTiledFn fn = []() -> EncodeTiledFn {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qr;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
         qr == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
+      return reinterpret_cast<EncodeTiledFn>(p);
+    return nullptr;
+  }();
   return fn;
 }
 
@@ -1356,10 +1274,9 @@ bool make_attn_tc_plan(const pvlm_attn_params& p, AttnTcPlan& plan) {
   plan.total_tiles = (long long)plan.tiles_per_item * p.Hkv * p.n_layers;
   plan.n_cta = (int)(plan.total_tiles < kNumSMs ? plan.total_tiles : kNumSMs);
   if (p.max_ctas > 0 && p.max_ctas < plan.n_cta) plan.n_cta = p.max_ctas;
-  if (const char* e = getenv("PVLM_TC_CTAS")) {     // test hook: fewer CTAs => longer tile runs and more segments per CTA
-    const int v = atoi(e);
-    if (v >= 1 && v < plan.n_cta) plan.n_cta = v;
-  }
+  // test switch: fewer CTAs => longer tile runs and more segments per CTA
+  const int opt_ctas = option_value(PVLM_OPT_ATTN_MAX_CTAS);
+  if (opt_ctas >= 1 && opt_ctas < plan.n_cta) plan.n_cta = opt_ctas;
   const long long per_cta = (plan.total_tiles + plan.n_cta - 1) / plan.n_cta;
   plan.seg_max = (int)((per_cta + plan.tiles_per_item - 1) / plan.tiles_per_item) + 1;
   size_t off = 0;
@@ -1390,10 +1307,6 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   {
     const int nsb = (512 - 2 * plan.nrp) / plan.nrp >= 4 ? 4 : (512 - 2 * plan.nrp) / plan.nrp;
     a.lookahead = nsb - 1;
-    if (const char* e = getenv("PVLM_TC_LOOKAHEAD")) {      // tuning hook
-      const int v = atoi(e);
-      if (v >= 1 && v <= nsb - 1) a.lookahead = v;
-    }
   }
   cudaMemsetAsync(a.status, 0, 4, s);
   if (p.prof_event_begin) cudaEventRecord((cudaEvent_t)p.prof_event_begin, s);

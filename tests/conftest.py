@@ -24,3 +24,18 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture
+def pvlm_option():
+    """set(name, value) flips a process-wide library switch for this test only."""
+    from paper_2603_19610_b200 import binding
+    saved = {}
+
+    def set_(name, value):
+        prev = binding.set_option(name, value)
+        saved.setdefault(name, prev)
+
+    yield set_
+    for name, prev in saved.items():
+        binding.set_option(name, prev)

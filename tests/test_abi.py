@@ -75,6 +75,16 @@ def test_workspace_queries_and_argument_errors_need_no_gpu():
     assert L.pvlm_verify_attn(C.byref(p), None) == 3                    # no workspace
     p.Hq = 41
     assert L.pvlm_verify_attn(C.byref(p), None) == 2                    # Hq % Hkv != 0
+    # a listed-mass-layers count out of range makes the workspace query answer 0 (never a wrapped size)
+    p.Hq = 40
+    p.mass = 4096
+    layers = (C.c_int * 9)(*range(9))
+    p.mass_layers = layers
+    for bad in (0, -3, 9):
+        p.n_mass_layers = bad
+        assert L.pvlm_verify_attn_workspace_bytes(C.byref(p)) == 0
+    p.n_mass_layers = 2
+    assert 0 < L.pvlm_verify_attn_workspace_bytes(C.byref(p)) < (1 << 30)
 
     a = binding.AcceptParams()
     a.batch, a.gamma, a.V = 1, 12, 152064
@@ -89,6 +99,17 @@ def test_workspace_queries_and_argument_errors_need_no_gpu():
     u.k = 10
     assert L.pvlm_uvprune_workspace_bytes(C.byref(u)) >= 400
     assert L.pvlm_uvprune_select_gather(C.byref(u), None) == 1          # no mass pointer
+
+    # the decision-only entry points
+    assert L.pvlm_select_from_scores(None, 100, 101, None, None, 0, None) == 1    # k > m
+    assert L.pvlm_select_from_scores(None, 100, 10, None, None, 0, None) == 1     # no scores
+    assert L.pvlm_accept_from_probs(None, None, None, 3, 4, 1, None, None) == 1   # fewer uniforms than tokens
+    assert L.pvlm_accept_from_probs(None, None, None, 5, 4, 1, 4096, None) == 1   # no probabilities
+    assert L.pvlm_accept_from_probs(None, None, None, 5, 4, 0, 4096, None) == 1   # empty batch
+    # process-wide switches: unknown option or negative value refused, previous value returned
+    assert L.pvlm_set_option(99, 1) == -1 and L.pvlm_set_option(0, -1) == -1
+    prev = L.pvlm_set_option(2, 7)
+    assert L.pvlm_set_option(2, prev) == 7
 
     # the step call checks every stage before it queues anything (so this needs no GPU either)
     sp = binding.StepParams()

@@ -54,6 +54,58 @@ def check_against_oracle(tl, dl, tok, u, temperature=1.0):
     return g, r
 
 
+@pytest.mark.parametrize("cid", [0, 1, 2, 3, 4])
+def test_accepted_length_from_the_oracles_probabilities(cid):
+    """The accept decision on its own (pvlm_accept_from_probs), fed the ORACLE's fp32 p(x_t), q(x_t): the accepted
+    length is bit-exact on every workload config, several steps each, and on the edges of the uniform's range."""
+    cfg = wl.CONFIGS[cid]
+    for step in range(3):
+        tl, dl, tok, u = wl.accept_inputs(cfg, step)
+        r = oracle_accept(tl, dl, tok, u)
+        p_d, q_d = torch.from_numpy(r["p_tok"]).cuda(), torch.from_numpy(r["q_tok"]).cuda()
+        assert int(binding.accept_from_probs(p_d, q_d, torch.from_numpy(u).cuda())) == r["n_accept"]
+        for edge in (0.0, 1.0 - 2.0 ** -24):                   # smallest and largest uniform there is
+            ue = np.full_like(u, edge)
+            want = oracle_accept(tl, dl, tok, ue)["n_accept"]
+            assert int(binding.accept_from_probs(p_d, q_d, torch.from_numpy(ue).cuda())) == want
+            if edge == 0.0:
+                assert want == cfg.gamma                       # u = 0 accepts every token with p > 0
+
+
+def test_accepted_length_from_probabilities_random_trials():
+    """1e5 random trials of the decision alone against the rule written out in numpy fp32 (one rounded multiply,
+    strict compare, first failure), a third of them placed ON the boundary u * q == p and one ulp either side."""
+    rng = np.random.default_rng(99)
+    B, gamma = 100_000, 6
+    q = rng.random((B, gamma)).astype(np.float32) * np.float32(0.9) + np.float32(1e-3)
+    u = wl.unit_uniforms(rng, (B, gamma + 1))
+    p = (q * rng.random((B, gamma)).astype(np.float32) * np.float32(2.5)).astype(np.float32)       # ratios in [0, 2.5)
+    on = rng.random((B, gamma)) < 1 / 3
+    uq = (u[:, :gamma] * q).astype(np.float32)
+    side = rng.integers(-1, 2, size=(B, gamma))
+    edge = np.where(side < 0, np.nextafter(uq, np.float32(-1)), np.where(side > 0, np.nextafter(uq, np.float32(2)), uq))
+    p = np.where(on, edge, p).astype(np.float32)
+    ok = (u[:, :gamma] * q).astype(np.float32) < p
+    want = np.where(ok.all(axis=1), gamma, np.argmin(ok, axis=1)).astype(np.int32)
+    got = binding.accept_from_probs(torch.from_numpy(p).cuda(), torch.from_numpy(q).cuda(), torch.from_numpy(u).cuda())
+    np.testing.assert_array_equal(got.cpu().numpy(), want)
+    assert 0 < (want == gamma).sum() < B and (want == 0).any()
+    # the oracle's trial routine agrees on the same decision when given logits whose softmax it computes itself
+    V = 16
+    tl = (1.5 * rng.standard_normal((gamma + 1, V))).astype(np.float32)
+    dl = (tl[:gamma] + 0.7 * rng.standard_normal((gamma, V))).astype(np.float32)
+    x = rng.integers(0, V, size=(B, gamma))
+    n_ref, _ = spec_accept_trials(tl, dl, x, u)
+    P, Q = softmax64(tl), softmax64(dl)
+    t_idx = np.arange(gamma)[None, :]
+    got = binding.accept_from_probs(torch.from_numpy(P[t_idx, x].astype(np.float32)).cuda(),
+                                    torch.from_numpy(Q[t_idx, x].astype(np.float32)).cuda(), torch.from_numpy(u).cuda())
+    np.testing.assert_array_equal(got.cpu().numpy(), n_ref)
+    # gamma = 0: nothing to test
+    z = torch.empty((3, 0), dtype=torch.float32, device="cuda")
+    assert binding.accept_from_probs(z, z, torch.zeros((3, 1), device="cuda")).tolist() == [0, 0, 0]
+
+
 def test_config0():
     tl, dl, tok, u = wl.accept_inputs(wl.CONFIGS[0])
     check_against_oracle(tl, dl, tok, u)

@@ -51,14 +51,28 @@ def test_config_end_to_end(cid):
     g_cur, g_ref = mass[1].cpu().numpy(), mass[0].cpu().numpy()
     np.testing.assert_array_equal(kept.cpu().numpy(), select_topk(score_fp32(g_cur, g_ref, 0, cfg.m), cfg.k_keep))
     np.testing.assert_array_equal(score.cpu().numpy(), score_fp32(g_cur, g_ref, 0, cfg.m))
-    # ... and end to end may differ from the oracle's only where a score sits within 1e-4 relative of the k-th score
+    # ... bit-exact from the ORACLE's fp32 scores through the scores-only entry point ...
     s_or = score_fp32(M_cur.astype(np.float32), M_ref.astype(np.float32), 0, cfg.m)
     idx_or = select_topk(s_or, cfg.k_keep)
+    np.testing.assert_array_equal(binding.select_from_scores(torch.from_numpy(s_or).cuda(), cfg.k_keep).cpu().numpy(), idx_or)
+    # ... and end to end may differ from the oracle's only where a score sits within 1e-4 relative of the k-th score.
+    # A score is a difference of two masses, so where it is much smaller than they are the masses' own error
+    # (measured in this run as eps, itself asserted <= 1e-4 above) can exceed that band: an index outside the band
+    # must lie within the cancellation bound eps * (cur + ref) of both scores involved.  Each is printed.
     diff = np.setxor1d(kept.cpu().numpy(), idx_or)
-    tau = np.sort(s_or)[::-1][cfg.k_keep - 1]
+    order = np.argsort(-s_or, kind="stable")
+    i_tau = int(order[cfg.k_keep - 1])
+    tau = float(s_or[i_tau])
+    eps = max(float(np.abs(g_cur - M_cur).max() / np.abs(M_cur).max()), float(np.abs(g_ref - M_ref).max() / np.abs(M_ref).max()),
+              float((np.abs(g_cur - M_cur) / np.abs(M_cur)).max()), float((np.abs(g_ref - M_ref) / np.abs(M_ref)).max()))
     for i in diff:
-        assert abs(float(s_or[i]) - float(tau)) <= 1e-4 * max(abs(float(s_or[i])), abs(float(tau)), 1e-30) + 2e-6, \
-            (i, s_or[i], tau)
+        gap = abs(float(s_or[i]) - tau)
+        band = 1e-4 * max(abs(float(s_or[i])), abs(tau), 1e-30)
+        if gap > band:
+            bound = eps * float(M_cur[i] + M_ref[i] + M_cur[i_tau] + M_ref[i_tau])
+            print(f"config {cid}: index {i} outside the relative band: |s - tau| = {gap:.3e}, band {band:.3e}, "
+                  f"cancellation bound {bound:.3e} (eps {eps:.2e})")
+            assert gap <= bound, (i, s_or[i], tau, gap, band, bound)
     assert diff.size <= max(4, cfg.k_keep // 100)
 
     # gather is byte exact for the indices the GPU selected
@@ -71,6 +85,10 @@ def test_config_end_to_end(cid):
 
     # accept / resample
     r = oracle_accept(tl, dl, tok, u)
+    # accepted length bit-exact from the ORACLE's fp32 probabilities through the probabilities-only entry point
+    n_from_oracle = binding.accept_from_probs(torch.from_numpy(r["p_tok"]).cuda(), torch.from_numpy(r["q_tok"]).cuda(),
+                                              torch.from_numpy(u).cuda())
+    assert int(n_from_oracle) == r["n_accept"]
     n_g = int(acc["n_accept"])
     if n_g != r["n_accept"]:
         t = min(n_g, r["n_accept"])

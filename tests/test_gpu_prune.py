@@ -97,10 +97,10 @@ def test_select_from_oracle_masses_config0():
     np.testing.assert_array_equal(kept, select_topk(score_fp32(cur, ref, 0, cfg.m), cfg.k_keep))
 
 
-def test_single_cta_kernels_still_match(monkeypatch):
-    """PVLM_SELECT_IMPL=cta keeps the selection on the single-CTA kernels (register-resident up to
+def test_single_cta_kernels_still_match(pvlm_option):
+    """The select_one_cta switch keeps the selection on the single-CTA kernels (register-resident up to
     32,768 scores, global-memory keys above): the second implementation of the same selection."""
-    monkeypatch.setenv("PVLM_SELECT_IMPL", "cta")
+    pvlm_option("select_one_cta", 1)
     rng = np.random.default_rng(77)
     for m, k in [(30720, 3072), (131072, 6553), (5000, 4999)]:
         cur = (np.round(rng.random(m) * 4096) / 4096).astype(np.float32)       # ties included

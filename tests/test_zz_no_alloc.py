@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle.uvprune import score_fp32, select_topk
 from paper_2603_19610_b200 import binding
 
 pytestmark = pytest.mark.gpu
@@ -35,6 +36,10 @@ def test_static_scratch_select_matches_workspace_select_twice_in_a_row():
         torch.cuda.synchronize()
         assert torch.equal(got_idx, want_idx)                                  # indices: bit-exact
         assert torch.equal(got_score, want_score)
+        # and both against the CPU oracle (score bits, kept indices)
+        s_ref = score_fp32(cur.cpu().numpy(), ref.cpu().numpy(), v0, m)
+        assert (got_score.cpu().numpy().view(np.uint32) == s_ref.view(np.uint32)).all()
+        np.testing.assert_array_equal(got_idx.cpu().numpy(), select_topk(s_ref, k))
     # raw-signal mode (no reference layer) and the empty selection
     cur, _ = _case(1000, 10, 0, 3, True)
     want_idx, _, _, _ = binding.uvprune_select_gather(cur, None, 0, 1000, 10)
@@ -42,6 +47,7 @@ def test_static_scratch_select_matches_workspace_select_twice_in_a_row():
     binding.uvprune_select_static(cur, None, 0, 1000, 10, got_idx)
     torch.cuda.synchronize()
     assert torch.equal(got_idx, want_idx)
+    np.testing.assert_array_equal(got_idx.cpu().numpy(), select_topk(cur.cpu().numpy()[:1000], 10))
     binding.uvprune_select_static(cur, None, 0, 1000, 0, torch.empty(0, dtype=torch.int32, device="cuda"))
 
 
