@@ -389,9 +389,24 @@ pvlm_status pvlm_acceptance_rate(const pvlm_rate_params *p, void *stream);
  * round runs, on `draft_stream`, the gamma draws from the draft rows
  * (pvlm_spec_accept with gamma = 0, batch = gamma) and, on `target_stream`,
  * the accept / reject / resample kernels over the tokens under test; if
- * target_attn / draft_attn are given, the round also runs that attention
- * call once on the target stream and gamma times on the draft stream as the
- * forwards' memory traffic (their outputs are not used).  Random numbers are
+ * target_attn / draft_attn are given, the round also runs the two models'
+ * attention over their caches as they stand in that round (the outputs are not
+ * used; the logit tables stand in for the rest of the forward):
+ *   target: one call with n_ctx = target_attn->n_ctx + (tokens committed so
+ *           far) and R = (tokens under test) + 1: the committed tokens have
+ *           become context, the window holds the last committed token and the
+ *           drafts being verified;
+ *   draft : gamma calls (R = 1), step t with n_ctx = draft_attn->n_ctx +
+ *           (tokens committed) + (drafts pending) + t: the draft's cache grows
+ *           by one row per token it writes, and after a rejection it is
+ *           truncated to the committed prefix (the replacement token is the
+ *           next step's input), so the next round starts from there.
+ * The blocks' n_ctx are the context lengths before the first generated token;
+ * their k / v must hold n_ctx + K + 2 * gamma + 1 token rows and their
+ * workspaces must cover every round's shape (sizing them with n_ctx + K +
+ * 2 * gamma and R = gamma + 1 does; a round whose call does not fit returns
+ * PVLM_ERR_WORKSPACE).  A bounded wait that expires inside one of these
+ * attention calls ends the loop with PVLM_ERR_TIMEOUT.  Random numbers are
  * indexed by round: u_draft[r][s] draws the s-th token drafted in round r,
  * u_accept[r][s] tests the s-th token verified in round r, u_resample[r]
  * draws round r's replacement.
@@ -402,6 +417,7 @@ pvlm_status pvlm_acceptance_rate(const pvlm_rate_params *p, void *stream);
  * sizes or NULL pointers PVLM_ERR_INVALID_ARG; P < K + 2*gamma + 1 or
  * max_rounds exhausted PVLM_ERR_TOO_LARGE; workspace as for the other calls.
  * ---------------------------------------------------------------------- */
+#define PVLM_DECODE_LOG_COLS 9
 typedef struct {
   const float *target_logits, *draft_logits;  /* fp32 [P][row_stride], first V of a row used */
   long long row_stride;                       /* elements, >= V                              */
@@ -411,8 +427,11 @@ typedef struct {
   const float *u_resample;                    /* fp32 [max_rounds]                            */
   int max_rounds;                             /* K rounds always suffice                      */
   int *tokens;                                /* HOST int32 [K] out                           */
-  int *round_log;                             /* HOST int32 [max_rounds][6] out, nullable:
-                                                 mode (0 Pre, 1 Post), verified, accepted, committed, dropped, start */
+  int *round_log;                             /* HOST int32 [max_rounds][PVLM_DECODE_LOG_COLS] out, nullable:
+                                                 mode (0 Pre, 1 Post), verified, accepted, committed, dropped, start,
+                                                 target_ctx, draft_ctx, draft_keep: generated tokens in the verification
+                                                 call's context, in the draft's cache before the round's first draft step,
+                                                 and in the draft's cache after the round's commit or rollback          */
   int *n_rounds;                              /* HOST int32 out, nullable                     */
   float *round_ms;                            /* HOST fp32 [max_rounds] out, nullable: device time of each round  */
   const pvlm_attn_params *target_attn;        /* HOST pointer to a complete block, nullable   */

@@ -80,9 +80,19 @@ class Schedule:
         return self.pending if (self.mode == POST and self.pending > 0) else 1
 
     def advance(self, n_accept: int) -> dict:
-        """Applies one round's verification outcome; returns what was committed and dropped."""
+        """Applies one round's verification outcome; returns what was committed and dropped, and the cache
+        lengths of the round, counted in rows beyond each model's context before the first generated token
+        (a model's forward takes its newest token as input, so a cache that "holds k generated tokens and
+        restarts from the next one" is k + 1 rows here):
+        target_ctx = context rows of the round's verification (the committed tokens; its window holds the last
+        committed token and the tokens under test); draft_ctx = context rows of the draft's first forward of the
+        round (committed and pending tokens); draft_keep = the same count after the round: everything the draft
+        has written if all was accepted, the committed prefix alone after a rejection (the cache rolls back and
+        the replacement token is the draft's next input)."""
         g = self.gamma
-        if self.mode == POST and self.pending > 0:
+        post = self.mode == POST and self.pending > 0
+        lengths = dict(target_ctx=self.committed, draft_ctx=self.committed + (self.pending if post else 0))
+        if post:
             nv = self.pending
             assert 0 <= n_accept <= nv
             if n_accept == nv:
@@ -104,6 +114,7 @@ class Schedule:
                 rec = dict(mode=PRE, verified=1, accepted=0, emitted=1, dropped=g, next_mode=PRE)
                 self.pending, self.mode = 0, PRE
         self.committed += rec["emitted"]
+        rec.update(lengths, draft_keep=self.committed + self.pending)
         self.log.append(rec)
         return rec
 
@@ -137,7 +148,8 @@ def parallel_decode(target_logits, draft_logits, gamma: int, K: int, u_draft, u_
     """Generates K tokens.  target_logits / draft_logits fp32 [P, V] with P >= K + 2 * gamma + 1 rows;
     u_draft, u_accept fp32 [rounds, gamma]; u_resample fp32 [rounds].
     Returns dict(tokens int32 [K], rounds, log (one record per round, as `Schedule.advance` plus
-    `start` = committed length at the round's start))."""
+    `start` = committed length at the round's start; the cache lengths target_ctx, draft_ctx, draft_keep of
+    `Schedule.advance` are checked against the token lists kept here))."""
     tl = np.asarray(target_logits, dtype=np.float32)
     dl = np.asarray(draft_logits, dtype=np.float32)
     q = softmax64(dl, temperature)
@@ -159,11 +171,13 @@ def parallel_decode(target_logits, draft_logits, gamma: int, K: int, u_draft, u_
         n = int(res["n_accept"])
         rec = s.advance(n)
         rec["start"] = L
+        assert rec["target_ctx"] == L and rec["draft_ctx"] == base      # the token lists and the schedule agree
         tokens.extend(int(x) for x in verify[:n])
         if n < nv:
             tokens.append(int(res["out_tokens"][n]))          # the replacement token
-            pending = []
+            pending = []                                      # rollback: the draft keeps the committed prefix only
         else:
             pending = fresh if post else fresh[1:]            # no bonus token: the draft has moved on
+        assert rec["draft_keep"] == len(tokens) + len(pending)
         r += 1
     return dict(tokens=np.asarray(tokens[:K], dtype=np.int32), rounds=r, log=s.log)

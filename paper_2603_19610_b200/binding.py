@@ -21,6 +21,7 @@ _LOCK = threading.Lock()
 STATUS_NAMES = {0: "PVLM_OK", 1: "PVLM_ERR_INVALID_ARG", 2: "PVLM_ERR_UNSUPPORTED",
                 3: "PVLM_ERR_WORKSPACE", 4: "PVLM_ERR_CUDA", 5: "PVLM_ERR_TOO_LARGE", 6: "PVLM_ERR_TIMEOUT"}
 SELECT_STATIC_MAX_M = 262144
+DECODE_LOG_COLS = 9
 
 
 class PvlmError(RuntimeError):
@@ -498,8 +499,9 @@ def parallel_decode(target_logits, draft_logits, gamma: int, K: int, u_draft, u_
     """The Pre-/Post-verify round loop on two streams (see pvlm_parallel_decode).
     target_logits / draft_logits fp32 [P, V] on the device (row i = distribution of generated position i),
     u_draft / u_accept fp32 [rounds, gamma], u_resample fp32 [rounds] on the device.  target_attn / draft_attn:
-    optional AttnParams blocks run as the forwards' traffic.  The target side uses the current stream.
-    Returns dict(tokens int32 [K], rounds, log int32 [rounds, 6], round_ms or None)."""
+    optional AttnParams blocks whose attention runs every round over the two caches as they stand (their n_ctx = context
+    before the first generated token; k / v and workspace must cover n_ctx + K + 2 * gamma + 1 rows).  The target side
+    uses the current stream.  Returns dict(tokens int32 [K], rounds, log int32 [rounds, DECODE_LOG_COLS], round_ms or None)."""
     _need_cuda(target_logits, draft_logits, u_draft, u_accept, u_resample)
     P, V = target_logits.shape
     assert draft_logits.shape == (P, V) and target_logits.stride(1) == 1 and draft_logits.stride(0) == target_logits.stride(0)
@@ -509,7 +511,7 @@ def parallel_decode(target_logits, draft_logits, gamma: int, K: int, u_draft, u_
     assert u_draft.shape == (max_rounds, gamma) and u_accept.shape == (max_rounds, gamma)
     ud, ua, ur = u_draft.contiguous(), u_accept.contiguous(), u_resample.contiguous()
     tokens = torch.empty(K, dtype=torch.int32)
-    log = torch.zeros((max_rounds, 6), dtype=torch.int32)
+    log = torch.zeros((max_rounds, DECODE_LOG_COLS), dtype=torch.int32)
     n_rounds = torch.zeros(1, dtype=torch.int32)
     ms = torch.zeros(max_rounds, dtype=torch.float32) if want_ms else None
     p = DecodeParams()

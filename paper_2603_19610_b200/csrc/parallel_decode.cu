@@ -1,8 +1,12 @@
 // Parallel decoding round loop (Algorithm 1: Pre-verify / Post-verify) on two CUDA streams.
 // The host side is the mode machine; every token is drawn, tested and replaced by the accept kernels.
+// The two models' caches are followed token by token: the verification call of a round sees the committed tokens
+// and the window under test, every draft step sees what the draft has written so far, and a rejection rolls the
+// draft's cache back to the committed prefix (appendix "Parallel Pipeline Details").
 #include "pvlm_common.cuh"
 
 #include <vector>
+#include <cstring>
 
 namespace pvlm {
 
@@ -117,9 +121,25 @@ pvlm_status pvlm_parallel_decode(const pvlm_decode_params* p, void* target_strea
   auto fail = [&](pvlm_status s) { if (st == PVLM_OK) st = s; };
   if (e != cudaSuccess) { set_cuda_error((int)e); fail(PVLM_ERR_CUDA); }
 
-  // host copies of one round's results: [n_accept | out_tokens (g+1) | fresh (g)]
-  std::vector<int> h_res(1 + (g + 1) + g), h_pending(g, 0);
+  // host copies of one round's results, in pinned memory (one small buffer per host thread, kept):
+  // [n_accept | out_tokens (g+1) | fresh (g) | status words: target, draft step 0..g-1]
+  static thread_local int* h_pinned = nullptr;
+  constexpr int kResWords = 1 + (kMaxGamma + 1) + kMaxGamma + 1 + kMaxGamma;
+  if (!h_pinned && cudaHostAlloc((void**)&h_pinned, kResWords * sizeof(int), cudaHostAllocDefault) != cudaSuccess) {
+    (void)cudaGetLastError();
+    h_pinned = nullptr;
+  }
+  std::vector<int> h_fallback(h_pinned ? 0 : kResWords), h_pending(g, 0);
+  int* h_res = h_pinned ? h_pinned : h_fallback.data();
+  int* h_status = h_res + 2 + 2 * g;                       // [0] target, [1 + t] draft step t
+  memset(h_res, 0, kResWords * sizeof(int));
   int mode = 0 /* Pre */, n_pending = 0, committed = 0, round = 0, cur = 0;
+  // Where a call's status word lives (a bounded wait inside the attention kernels that expired sets it).
+  auto status_word = [](const pvlm_attn_params& ap) -> const int* {
+    AttnPlan plan;
+    if (!make_attn_plan(ap, plan) || !plan.use_tc) return nullptr;
+    return reinterpret_cast<const int*>(static_cast<const char*>(ap.workspace) + plan.off_tc + plan.tc.off_status);
+  };
 
   while (st == PVLM_OK && committed < p->K) {
     if (round >= p->max_rounds) { fail(PVLM_ERR_TOO_LARGE); break; }
@@ -150,9 +170,15 @@ pvlm_status pvlm_parallel_decode(const pvlm_decode_params* p, void* target_strea
       const pvlm_status s2 = pvlm_spec_accept(&c, ds);
       if (s2 != PVLM_OK) { fail(s2); break; }
       if (!p->serial) e = cudaEventRecord(ev_drafted, ds);
+      // the draft's forwards: step t reads the cache as it stands after the tokens written so far
+      // (compacted context, committed tokens, pending drafts, this round's first t drafts) and adds one row
       for (int i = 0; i < g && p->draft_attn && st == PVLM_OK; ++i) {
-        const pvlm_status s3 = pvlm_verify_attn(p->draft_attn, ds);
-        if (s3 != PVLM_OK) fail(s3);
+        pvlm_attn_params da = *p->draft_attn;
+        da.n_ctx = p->draft_attn->n_ctx + base + i;
+        const pvlm_status s3 = pvlm_verify_attn(&da, ds);
+        if (s3 != PVLM_OK) { fail(s3); break; }
+        if (const int* w = status_word(da)) e = cudaMemcpyAsync(h_status + 1 + i, w, 4, cudaMemcpyDeviceToHost, ds);
+        if (e != cudaSuccess) break;
       }
       if (!p->serial && e == cudaSuccess) e = cudaEventRecord(ev_draft_done, ds);
       if (e != cudaSuccess) { set_cuda_error((int)e); fail(PVLM_ERR_CUDA); }
@@ -160,9 +186,16 @@ pvlm_status pvlm_parallel_decode(const pvlm_decode_params* p, void* target_strea
     }
 
     // ---- target side: the target forward's traffic, then accept / reject / resample over the tokens under test ----
+    // the target's forward: the committed tokens are context, the window holds the last committed token and the
+    // nv tokens under test
     if (p->target_attn) {
-      const pvlm_status s3 = pvlm_verify_attn(p->target_attn, ts);
+      pvlm_attn_params ta = *p->target_attn;
+      ta.n_ctx = p->target_attn->n_ctx + L;
+      ta.R = nv + 1;
+      const pvlm_status s3 = pvlm_verify_attn(&ta, ts);
       if (s3 != PVLM_OK) { fail(s3); break; }
+      if (const int* w = status_word(ta)) e = cudaMemcpyAsync(h_status, w, 4, cudaMemcpyDeviceToHost, ts);
+      if (e != cudaSuccess) { set_cuda_error((int)e); fail(PVLM_ERR_CUDA); break; }
     }
     if (!post && !p->serial) e = cudaStreamWaitEvent(ts, ev_drafted, 0);     // Pre-verify tests this round's first draft
     if (e != cudaSuccess) { set_cuda_error((int)e); fail(PVLM_ERR_CUDA); break; }
@@ -186,9 +219,9 @@ pvlm_status pvlm_parallel_decode(const pvlm_decode_params* p, void* target_strea
     // ---- join, read the round's outcome ----
     if (!p->serial) e = cudaStreamWaitEvent(ts, ev_draft_done, 0);
     if (e == cudaSuccess && p->round_ms) e = cudaEventRecord(ev_t1, ts);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(h_res.data(), sc.n_accept, 4, cudaMemcpyDeviceToHost, ts);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(h_res.data() + 1, sc.out_tokens, (size_t)(nv + 1) * 4, cudaMemcpyDeviceToHost, ts);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(h_res.data() + 2 + g, fresh, (size_t)g * 4, cudaMemcpyDeviceToHost, ts);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h_res, sc.n_accept, 4, cudaMemcpyDeviceToHost, ts);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h_res + 1, sc.out_tokens, (size_t)(nv + 1) * 4, cudaMemcpyDeviceToHost, ts);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h_res + 2 + g, fresh, (size_t)g * 4, cudaMemcpyDeviceToHost, ts);
     if (e == cudaSuccess) e = cudaStreamSynchronize(ts);
     if (e != cudaSuccess) { set_cuda_error((int)e); fail(PVLM_ERR_CUDA); break; }
     if (p->round_ms) {
@@ -197,9 +230,15 @@ pvlm_status pvlm_parallel_decode(const pvlm_decode_params* p, void* target_strea
       p->round_ms[round] = ms;
     }
 
+    // a bounded wait that expired inside one of this round's attention calls: its outputs are undefined
+    {
+      int any = h_status[0];
+      for (int i = 0; i < g; ++i) any |= h_status[1 + i];
+      if (any) { fail(PVLM_ERR_TIMEOUT); break; }
+    }
     // ---- the mode machine ----
     const int n = h_res[0];
-    const int* h_fresh = h_res.data() + 2 + g;
+    const int* h_fresh = h_res + 2 + g;
     if (n < 0 || n > nv) { fail(PVLM_ERR_CUDA); break; }
     int emitted, dropped, next_mode, next_pending;
     auto commit = [&](int tok) { if (committed < p->K) p->tokens[committed] = tok; ++committed; };
@@ -216,8 +255,11 @@ pvlm_status pvlm_parallel_decode(const pvlm_decode_params* p, void* target_strea
       emitted = 1; dropped = 0; next_pending = g - 1; next_mode = next_pending > 0 ? 1 : 0;
     }
     if (p->round_log) {
-      int* r = p->round_log + (long long)round * 6;
+      int* r = p->round_log + (long long)round * PVLM_DECODE_LOG_COLS;
       r[0] = post ? 1 : 0; r[1] = nv; r[2] = n; r[3] = emitted; r[4] = dropped; r[5] = L;
+      r[6] = L;                              // generated tokens in the verification call's context
+      r[7] = base;                           // generated tokens in the draft's cache before its first step of the round
+      r[8] = L + emitted + next_pending;     // ... and after the round: a rejection truncates it to the committed prefix
     }
     for (int i = 0; i < g; ++i) h_pending[i] = h_fresh[i];      // tail [g - next_pending, g) is what stays pending
     mode = next_mode;

@@ -1,5 +1,7 @@
 """Parity of pvlm_parallel_decode (Algorithm 1 on two streams) with the pipeline oracle: committed tokens and
-the per-round log (mode, verified, accepted, committed, dropped, start) must be identical."""
+the per-round log (mode, verified, accepted, committed, dropped, start, and the three cache lengths: tokens in the
+verification's context, in the draft's cache before the round, in the draft's cache after commit / rollback) must be
+identical."""
 import numpy as np
 import pytest
 import torch
@@ -26,7 +28,8 @@ def gpu_decode(tl, dl, gamma, K, ud, ua, ur, **kw):
 
 
 def log_rows(log):
-    return [[r["mode"], r["verified"], r["accepted"], r["emitted"], r["dropped"], r["start"]] for r in log]
+    return [[r["mode"], r["verified"], r["accepted"], r["emitted"], r["dropped"], r["start"],
+             r["target_ctx"], r["draft_ctx"], r["draft_keep"]] for r in log]
 
 
 @pytest.mark.parametrize("V,K,gamma,sigma,seed", [(50, 40, 4, 0.8, 3), (1000, 64, 9, 0.5, 7), (4099, 33, 1, 0.7, 11),
@@ -48,21 +51,47 @@ def test_serial_order_and_attention_payloads_do_not_change_the_tokens():
     ref = oracle_decode(tl, dl, gamma, K, ud, ua, ur)
     ser = gpu_decode(tl, dl, gamma, K, ud, ua, ur, serial=True)
     np.testing.assert_array_equal(ser["tokens"].numpy(), ref["tokens"])
-    # forwards' traffic: a target verification over a 3000-token context and a draft decode step over 400 tokens
+    # the two models' attention over their caches: a target context of 3000 tokens, a compacted draft context of 400;
+    # every round's calls follow the caches (committed tokens become context, the draft's cache grows and rolls back)
     dev = torch.device("cuda")
     mk = lambda *s: torch.randn(s, device=dev, dtype=torch.float32).to(torch.bfloat16)
     R = gamma + 1
-    qt, kt, vt = mk(2, R, 8, 128), mk(2, 3000 + R, 2, 128), mk(2, 3000 + R, 2, 128)
-    qd, kd, vd = mk(2, 1, 8, 128), mk(2, 401, 2, 128), mk(2, 401, 2, 128)
+    rows_t, rows_d = 3000 + K + 2 * gamma + 1, 400 + K + 2 * gamma + 1
+    qt, kt, vt = mk(2, R, 8, 128), mk(2, rows_t, 2, 128), mk(2, rows_t, 2, 128)
+    qd, kd, vd = mk(2, 1, 8, 128), mk(2, rows_d, 2, 128), mk(2, rows_d, 2, 128)
     ws_t = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
     ws_d = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
-    pt = binding.attn_params(qt, kt, vt, 3000, torch.empty_like(qt), None, None, workspace=ws_t)
-    pd = binding.attn_params(qd, kd, vd, 400, torch.empty_like(qd), None, None, workspace=ws_d)
+    pt = binding.attn_params(qt, kt[:, :3000 + R], vt[:, :3000 + R], 3000, torch.empty_like(qt), None, None, workspace=ws_t)
+    pd = binding.attn_params(qd, kd[:, :401], vd[:, :401], 400, torch.empty_like(qd), None, None, workspace=ws_d)
     out = gpu_decode(tl, dl, gamma, K, ud, ua, ur, target_attn=pt, draft_attn=pd, want_ms=True)
     np.testing.assert_array_equal(out["tokens"].numpy(), ref["tokens"])
     assert out["log"].tolist() == log_rows(ref["log"])
     assert out["round_ms"].shape[0] == out["rounds"] and float(out["round_ms"].min()) > 0.0
     assert binding.lib().pvlm_verify_attn_check(binding.C.byref(pt), None) == 0
+
+
+def test_cache_lengths_follow_commit_and_rollback():
+    """The logged cache lengths against their definition, round by round: the verification's context is what is
+    committed; the draft starts a round with the committed and pending tokens in its cache, ends it with gamma more,
+    and keeps either all of them (everything accepted) or the committed prefix alone (a rejection: the replacement
+    token is not in the cache yet, it is the next forward's input)."""
+    V, K, gamma = 500, 120, 5
+    tl, dl, ud, ua, ur = make_case(V, K, gamma, 0.7, 33)
+    out = gpu_decode(tl, dl, gamma, K, ud, ua, ur)
+    log = out["log"].tolist()
+    committed, pending, rollbacks = 0, 0, 0
+    for mode, verified, accepted, emitted, dropped, start, t_ctx, d_ctx, d_keep in log:
+        assert start == committed == t_ctx
+        assert d_ctx == committed + (pending if mode == 1 else 0)
+        committed += emitted
+        if accepted < verified:
+            pending = 0
+            rollbacks += 1
+            assert d_keep == committed and d_keep < d_ctx + gamma          # the cache was truncated
+        else:
+            pending = gamma if mode == 1 else gamma - 1
+            assert d_keep == committed + pending == d_ctx + gamma          # nothing dropped
+    assert rollbacks > 3 and committed >= K
 
 
 def test_argument_errors():

@@ -14,28 +14,61 @@ GOLD = os.path.join(os.path.dirname(__file__), "golden")
 
 
 def test_worked_example_of_the_appendix():
-    cfg, rounds = {}, []
+    cfg, rounds, cache_after = {}, [], {}
     for line in open(os.path.join(GOLD, "pipeline_example.txt")):
         if line.startswith("#") or not line.strip():
             continue
         parts = line.split()
         if parts[0] == "round":
             rounds.append(tuple(int(x) for x in parts[1:3] + parts[4:6]))
+        elif parts[0] == "draft_cache_after_round":
+            cache_after[int(parts[1])] = int(parts[2])
         else:
             cfg[parts[0]] = int(parts[1])
     s = Schedule(cfg["gamma"], cfg["start_mode"], cfg["start_pending"], cfg["start_committed"])
     run, longest = cfg["start_committed"], 0            # the pre-verified first token opens the run
-    for verified, accepted, committed, next_mode in rounds:
+    for i, (verified, accepted, committed, next_mode) in enumerate(rounds, start=1):
         assert s.n_verify() == verified
+        before = s.committed
         rec = s.advance(accepted)
         assert (rec["emitted"], rec["next_mode"]) == (committed, next_mode)
+        # cache lengths: the verification's context is what was committed; the draft keeps one row per generated
+        # token it restarts AFTER, so "k generated tokens stay in its cache" reads draft_keep = k + 1
+        assert rec["target_ctx"] == before
+        if i in cache_after:
+            assert rec["draft_keep"] - 1 == cache_after[i] and accepted < verified
+        else:
+            assert rec["draft_keep"] == rec["draft_ctx"] + cfg["gamma"]          # nothing dropped: gamma more rows
         run += accepted
         longest = max(longest, run)
         if accepted < verified:
             run = 0
+    assert len(cache_after) == 2
     assert s.committed == cfg["total_committed"] and len(s.log) == cfg["total_rounds"]
     assert len(s.log) * max(cfg["gamma"], cfg["gamma"]) == cfg["total_time_in_t"]      # c = gamma: a round lasts 3t
     assert longest == cfg["longest_accepted_run"]
+
+
+def test_round_sequence_from_a_pre_verify_start_under_this_builds_reading():
+    """The mode machine started in Pre-verify mode, against a hand-written round table that records this build's
+    READING of the Pre -> Post transition (gamma - 1 drafts stay pending); the fixture says so itself."""
+    gamma, rounds, total = None, [], None
+    for line in open(os.path.join(GOLD, "pipeline_from_pre_reading.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        parts = line.split()
+        if parts[0] == "gamma":
+            gamma = int(parts[1])
+        elif parts[0] == "total_committed":
+            total = int(parts[1])
+        else:
+            rounds.append(tuple(int(x) for x in parts[1:4] + parts[5:9]))
+    s = Schedule(gamma)
+    for mode, verified, accepted, committed, dropped, next_mode, pending_after in rounds:
+        assert (s.mode if s.pending else PRE, s.n_verify()) == (mode, verified)
+        rec = s.advance(accepted)
+        assert (rec["mode"], rec["emitted"], rec["dropped"], rec["next_mode"], s.pending) == (mode, committed, dropped, next_mode, pending_after)
+    assert s.committed == total
 
 
 def test_closed_forms_and_their_stated_consequences():
