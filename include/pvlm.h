@@ -329,6 +329,11 @@ typedef struct {
    * copy_stream behind them, and o is downloaded on copy_stream while select/gather run.  The call still
    * orders everything so that synchronising `stream` alone is enough afterwards. */
   void *copy_stream, *event_a, *event_b;
+  /* Optional HOST int32 [1] (NULL = off): receives the status word of the attention stage (of the last attention call
+   * on attn.workspace if run_attn is 0) with the other results: 0 = fine, non-zero = a bounded wait inside its kernels
+   * expired and o, mass and everything computed from them (kept_idx, the gathered cache) are undefined for this step.
+   * Without it, call pvlm_verify_attn_check(&attn, stream) after the stream has been synchronised to learn the same. */
+  int *h_attn_status;
 } pvlm_step_params;
 
 pvlm_status pvlm_verify_step(const pvlm_step_params *p, void *stream);

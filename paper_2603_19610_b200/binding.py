@@ -81,7 +81,8 @@ class StepParams(C.Structure):
                 ("h_draft_tokens", C.c_void_p), ("h_uniforms", C.c_void_p),
                 ("h_o", C.c_void_p), ("h_n_accept", C.c_void_p), ("h_out_tokens", C.c_void_p),
                 ("h_kept_idx", C.c_void_p),
-                ("copy_stream", C.c_void_p), ("event_a", C.c_void_p), ("event_b", C.c_void_p)]
+                ("copy_stream", C.c_void_p), ("event_a", C.c_void_p), ("event_b", C.c_void_p),
+                ("h_attn_status", C.c_void_p)]
 
 
 class DecodeParams(C.Structure):
@@ -362,7 +363,7 @@ def verify_step(attn: AttnParams | None, prune: PruneParams | None, accept: Acce
     attn / prune / accept are parameter blocks built by attn_params / prune_params /
     accept_params (None skips the stage).  host_in maps h_q, h_k_window, h_v_window,
     h_target_logits, h_draft_logits, h_draft_tokens, h_uniforms to (pinned) CPU tensors
-    copied to the device first; host_out maps h_o, h_n_accept, h_out_tokens, h_kept_idx to
+    copied to the device first; host_out maps h_o, h_n_accept, h_out_tokens, h_kept_idx, h_attn_status to
     CPU tensors filled at the end.  overlap = (torch.cuda.Stream, torch.cuda.Event, torch.cuda.Event)
     lets the library overlap the accept-input upload and the output download with compute (the
     events must have been recorded once so that their handles exist).

@@ -368,7 +368,6 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     if (p->h_out_tokens && ok())
       e = cudaMemcpyAsync(p->h_out_tokens, c.out_tokens, (size_t)c.batch * (c.gamma + 1) * 4, cudaMemcpyDeviceToHost, cs);
   }
-  if ((accept_on_side || split_gather) && ok()) e = cudaEventRecord(ea, cs);   // the side stream's stages are complete after this
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   if (p->run_attn && p->h_o) {                                   // o is final: its download may overlap the rest
     const size_t q_layer = (size_t)a.R * a.Hq * a.D * 2;
@@ -377,8 +376,13 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
       if (ok()) e = cudaStreamWaitEvent(cs, eb, 0);
     }
     if (ok()) e = cudaMemcpy2DAsync(p->h_o, q_layer, a.o, (size_t)a.q_layer_stride * 2, q_layer, a.n_layers, cudaMemcpyDeviceToHost, cs);
-    if (overlap && ok()) e = cudaEventRecord(eb, cs);
     if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
+  }
+  if (p->h_attn_status) {          // did a bounded wait inside the attention kernels (this step's, or the last call's) expire?
+    AttnPlan plan;
+    *p->h_attn_status = 0;
+    if (a.workspace && make_attn_plan(a, plan) && plan.use_tc && a.workspace_bytes >= plan.total && ok())
+      e = cudaMemcpyAsync(p->h_attn_status, (const char*)a.workspace + plan.off_tc + plan.tc.off_status, 4, cudaMemcpyDeviceToHost, s);
   }
   if (p->run_prune) {
     st = split_gather ? launch_uvprune_parts(p->prune, true, 2, s) : pvlm_uvprune_select_gather(&p->prune, stream);
@@ -392,8 +396,10 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     e = cudaMemcpyAsync(p->h_n_accept, c.n_accept, (size_t)c.batch * 4, cudaMemcpyDeviceToHost, s);
   if (p->run_accept && !accept_on_side && p->h_out_tokens && ok())
     e = cudaMemcpyAsync(p->h_out_tokens, c.out_tokens, (size_t)c.batch * (c.gamma + 1) * 4, cudaMemcpyDeviceToHost, s);
-  if ((accept_on_side || split_gather) && ok()) e = cudaStreamWaitEvent(s, ea, 0);   // `stream` now also covers the side stream's stages
-  if (overlap && p->run_attn && p->h_o && ok()) e = cudaStreamWaitEvent(s, eb, 0);   // `stream` now also covers the o download
+  // The side stream was forked from `stream` at the top; whatever was (or was not) queued on it, it is joined back
+  // here, so that synchronising `stream` alone covers everything and a stream capture of the call always closes.
+  if (overlap && ok()) e = cudaEventRecord(ea, cs);
+  if (overlap && ok()) e = cudaStreamWaitEvent(s, ea, 0);
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   return PVLM_OK;
 }

@@ -250,6 +250,43 @@ def test_timeout_status_is_reported_from_the_workspace_word():
     assert binding.lib().pvlm_verify_attn_check(C.byref(p), st) == 0
 
 
+def test_first_attention_calls_from_two_host_threads_at_once():
+    """Two host threads make their FIRST call into the library at the same moment (a fresh process, so the one-time
+    look-ups inside the first call really race); both must succeed and give what a later single call gives."""
+    import os
+    import subprocess
+    import sys
+    prog = r"""
+import sys, threading, numpy as np, torch
+sys.path.insert(0, %r)
+from paper_2603_19610_b200 import binding, workloads as wl
+binding.lib()                                         # load (and if need be build) the library before the race
+dev = torch.device("cuda")
+to_dev = lambda b: torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).to(dev)
+cases = [tuple(to_dev(x) for x in wl.make_qkv(8, 2, 128, 3, 1003, True, seed=s)) for s in (1, 2)]
+gate, out, err = threading.Barrier(2), [None, None], []
+def work(i):
+    try:
+        with torch.cuda.stream(torch.cuda.Stream()):
+            q, k, v = cases[i]
+            gate.wait()
+            out[i] = binding.verify_attn(q, k, v, 1000, want_mass=True, check=True)
+    except Exception as e:                            # noqa: BLE001
+        err.append(repr(e))
+ts = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+[t.start() for t in ts]; [t.join() for t in ts]
+torch.cuda.synchronize()
+assert not err, err
+for i in range(2):
+    want = binding.verify_attn(*cases[i], 1000, want_mass=True, check=True)
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip(out[i], want))
+print("ok")
+""" % os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-c", prog], capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0 and res.stdout.strip().endswith("ok"), res.stdout[-2000:] + res.stderr[-2000:]
+
+
 def test_tensor_core_path_is_deterministic():
     """Same inputs twice through the tcgen05 kernels: bitwise equal O, lse and mass (no float atomics,
     fixed-order merges)."""

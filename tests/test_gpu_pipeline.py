@@ -299,6 +299,61 @@ def test_the_three_calls_replay_from_a_cuda_graph(cid):
     assert int(got[6]) == r["n_accept"]
 
 
+def test_step_call_reports_the_attention_status_word():
+    """The status word of the attention stage comes back with the step's other host results.  No GPU wait is made
+    to expire: the word is poisoned from the host after a clean call and read back through a step that runs no stage."""
+    qb, kb, vb = wl.make_qkv(8, 2, 128, 3, 303, sink=False, seed=3)
+    q, k, v = bf16_cuda(qb), bf16_cuda(kb), bf16_cuda(vb)
+    pa = binding.attn_params(q, k, v, 300, torch.empty_like(q), None, None)
+    status = torch.full((1,), 77, dtype=torch.int32).pin_memory()
+    binding.verify_step(pa, None, None, host_out=dict(h_attn_status=status))
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    need = binding.lib().pvlm_verify_attn_workspace_bytes(C.byref(pa))
+    pa._keep[6][need - 8192:need - 8188] = torch.tensor([1, 0, 0, 0], dtype=torch.uint8, device="cuda")
+    sp = binding.StepParams()
+    sp.attn = pa
+    sp.h_attn_status = C.c_void_p(status.data_ptr())
+    assert binding.lib().pvlm_verify_step(C.byref(sp), C.c_void_p(torch.cuda.current_stream().cuda_stream)) == 0
+    torch.cuda.synchronize()
+    assert int(status[0]) == 1
+    binding.verify_step(pa, None, None, host_out=dict(h_attn_status=status))          # a new attention call clears it
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+
+
+def test_step_call_with_an_idle_side_stream_is_capturable():
+    """Overlap handles given but nothing for the side stream to do (attention only, select without a gather):
+    the side stream is still joined back, so a stream capture of the call closes and replays."""
+    cfg = wl.CONFIGS[0]
+    ref_in, cur_in = layers_for(cfg)
+    q = torch.stack([bf16_cuda(ref_in[0]), bf16_cuda(cur_in[0])])
+    k = torch.stack([bf16_cuda(ref_in[1]), bf16_cuda(cur_in[1])])
+    v = torch.stack([bf16_cuda(ref_in[2]), bf16_cuda(cur_in[2])])
+    o = torch.empty_like(q)
+    mass = torch.empty((2, cfg.T), dtype=torch.float32, device="cuda")
+    kept = torch.empty(cfg.k_keep, dtype=torch.int32, device="cuda")
+    s, side = torch.cuda.Stream(), torch.cuda.Stream()
+    evs = [torch.cuda.Event(), torch.cuda.Event()]
+    for e in evs:
+        e.record()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        pa = binding.attn_params(q, k, v, cfg.n_ctx, o, None, mass, mass_layers=[0, 1])
+        pp = binding.prune_params(mass[1], mass[0], 0, cfg.m, cfg.k_keep, kept, None, None, None, None, None)
+        for blocks in ((pa, None), (pa, pp)):
+            binding.verify_step(blocks[0], blocks[1], None, overlap=(side, evs[0], evs[1]))      # warm-up, direct
+            torch.cuda.synchronize()
+            want = (o.clone(), mass.clone(), kept.clone())
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                binding.verify_step(blocks[0], blocks[1], None, overlap=(side, evs[0], evs[1]))
+            o.zero_(); mass.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(o, want[0]) and torch.equal(mass, want[1]) and torch.equal(kept, want[2])
+
+
 def test_similarity_and_acceptance_rate_replay_from_a_cuda_graph():
     """The hidden-state criterion (three kernels chained by programmatic dependent launch) and the acceptance-rate
     pass are capturable too: a replay equals the direct calls bit for bit."""
