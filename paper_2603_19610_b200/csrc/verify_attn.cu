@@ -410,7 +410,9 @@ bool make_attn_plan(const pvlm_attn_params& p, AttnPlan& plan) {
   if (p.mass) {
     if (p.mass_layers && (p.n_mass_layers < 1 || p.n_mass_layers > 8)) return false;
     const int n_mass = p.mass_layers ? p.n_mass_layers : p.n_layers;
-    off += align_up((size_t)n_mass * p.Hkv * align_up(plan.T, kAttnBN) * 4, 256);
+    // per-KV-head partial sums; two per head where the tensor-core mass pass splits the query rows between its groups
+    const int parts = (plan.rows_pad == 96 || plan.rows_pad == 128) ? 2 : 1;
+    off += align_up((size_t)n_mass * p.Hkv * parts * align_up(plan.T, kAttnBN) * 4, 256);
   }
   // main pass on the tcgen05 kernel whenever it applies (PVLM_ATTN_IMPL=mma forces the mma.sync kernel)
   const bool force_mma = option_value(PVLM_OPT_ATTN_MMA_SYNC) != 0;

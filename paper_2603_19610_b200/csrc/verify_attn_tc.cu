@@ -47,7 +47,10 @@ constexpr int kTileBytes = 2 * kBoxBytes;  // 32 KB
 constexpr int kSoftmaxThreads = 256;
 constexpr int kGroupThreads = 128;         // one softmax group
 constexpr int kThreads = 128 + kSoftmaxThreads;   // warpgroup 0: TMA + MMA (+2 idle warps); warpgroups 1, 2: softmax
-constexpr uint32_t kSuspendHintNs = 20000;        // upper bound of one sleep inside try_wait
+#ifndef PVLM_SUSPEND_NS
+#define PVLM_SUSPEND_NS 20000
+#endif
+constexpr uint32_t kSuspendHintNs = PVLM_SUSPEND_NS;        // upper bound of one sleep inside try_wait
 constexpr uint64_t kWaitLimitNs = 1000000000ull;   // a wait that lasts a second has failed
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 constexpr float kNegBig = -1.0e30f;        // "no key seen yet" reference: finite, so differences never give NaN
@@ -213,19 +216,29 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
 // K and V tiles share one ring of 32 KB slots, filled and drained in the order the issuer consumes them.
 // Five slots fit beside Q and the two P buffers up to 80 padded rows.
 __host__ __device__ constexpr int ring_slots(int nrp) { return nrp <= 80 ? 5 : nrp <= 112 ? 4 : 3; }
-__host__ __device__ constexpr int s_bufs(int nrp) { return (512 - 2 * nrp) / nrp >= 4 ? 4 : (512 - 2 * nrp) / nrp; }
+// Wide row groups (96 or 128 padded rows) run in SPLIT-COLUMN mode: both softmax groups work on EVERY tile, each on
+// half of the query-row columns, instead of on alternate tiles.  A thread then holds half as many scores and running
+// row sums (2 x 48 or 2 x 64 registers instead of 2 x 96 / 2 x 128, which spilled), there is one output accumulator
+// and one partial per segment instead of two, and the freed TMEM columns hold one more score buffer.
+__host__ __device__ constexpr bool split_cols(int nrp) { return nrp == 96 || nrp == 128; }
+__host__ __device__ constexpr int s_bufs(int nrp) {
+  return split_cols(nrp) ? ((512 - nrp) / nrp >= 4 ? 4 : (512 - nrp) / nrp)
+                         : ((512 - 2 * nrp) / nrp >= 4 ? 4 : (512 - 2 * nrp) / nrp);
+}
 
 // HT: the last 16-column chunk holds at most 8 real query rows, so only its first 8 columns are processed.
 template <int NRP, bool HT>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const TcArgs a) {
-  constexpr int NCH = NRP / 16;            // 16-column chunks per thread
+  constexpr bool SC = split_cols(NRP);     // both groups on every tile, half of the columns each
+  constexpr int NCH = SC ? NRP / 32 : NRP / 16;            // 16-column chunks per thread
+  static_assert(!(SC && HT), "split-column mode processes whole chunks");
   auto CW = [](int c) constexpr { return (HT && c == NRP / 16 - 1) ? 8 : 16; };   // processed columns of chunk c
   constexpr int QBOX = NRP * 128;          // bytes of one 64-channel box of Q
   constexpr int PBYTES = NRP * 256;        // one P buffer: NRP/8 row groups x 2048 B
   constexpr int NSB = s_bufs(NRP);         // score buffers in TMEM
   constexpr int NS = ring_slots(NRP);      // K/V ring slots
-  constexpr uint32_t NEED = (2 + NSB) * NRP;
+  constexpr uint32_t NEED = ((SC ? 1 : 2) + NSB) * NRP;
   constexpr uint32_t TMEM_COLS = NEED <= 32 ? 32 : NEED <= 64 ? 64 : NEED <= 128 ? 128 : NEED <= 256 ? 256 : 512;
   constexpr uint32_t IDESC_QK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NRP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   constexpr uint32_t IDESC_PV = IDESC_QK | (1u << 15) | (1u << 16);
@@ -260,7 +273,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int item_first = (int)(f_begin / Tt);
 
   if (tid == 0) {
-    for (int i = 0; i < 4; ++i) { mbar_init(bar(K_FULL + i), 1); mbar_init(bar(P_FULL + i), kGroupThreads + 1); }
+    for (int i = 0; i < 4; ++i) { mbar_init(bar(K_FULL + i), 1); mbar_init(bar(P_FULL + i), (SC ? kSoftmaxThreads : kGroupThreads) + 1); }
     for (int i = 0; i < 2; ++i) mbar_init(bar(P_FREE + i), 1);
     for (int i = 0; i < NSB; ++i) mbar_init(bar(S_FULL + i), 1);
     for (int i = 0; i < NS; ++i) mbar_init(bar(EMPTY + i), 1);
@@ -283,7 +296,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
   const uint32_t tmem_O = tmem;                    // O accumulators of the two softmax groups: columns [g*NRP, (g+1)*NRP)
-  const uint32_t tmem_S = tmem + 2 * NRP;          // score buffers
+  const uint32_t tmem_S = tmem + (SC ? 1 : 2) * NRP;   // score buffers (split-column mode has one accumulator)
 
   if (f_end > f_begin) {
     if (warp < 4) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
@@ -381,8 +394,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             if (!wait_all(bar(P_FULL + (j & 3)), (j >> 2) & 1)) { ok = false; break; }     // P stored and V landed
             tc_fence_after();
             const uint64_t dv = desc_v0 + (uint64_t)((slot * kTileBytes) >> 4), dp = desc_p0 + (uint64_t)((g * PBYTES) >> 4);
-            const uint32_t d_tmem = tmem_O + g * NRP;
-            const uint32_t acc0 = i >= 2;                  // each group's accumulator starts afresh in every segment
+            const uint32_t d_tmem = tmem_O + (SC ? 0 : g * NRP);
+            const uint32_t acc0 = i >= (SC ? 1 : 2);       // each accumulator starts afresh in every segment
             if (elect_one()) {
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk)
@@ -410,13 +423,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const int t = q4 * 32 + lane;            // key within the tile == TMEM lane; channel d in the epilogue
       const int st = tid - 128;                // 0..255
       const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
-      float* m_s = s_m + g * 128;
-      float* fac_s = s_fac + g * 128;
-      int* newmax_s = s_newmax + g * 128;
+      constexpr int NR = NCH * 16;             // query-row columns this thread handles
+      const int r0 = SC ? g * NR : 0;          // the first of them (split-column mode: group 1 takes the upper half)
+      // per-row state: one set per group, or one set indexed by absolute row in split-column mode
+      float* m_s = s_m + (SC ? 0 : g * 128);
+      float* fac_s = s_fac + (SC ? 0 : g * 128);
+      int* newmax_s = s_newmax + (SC ? 0 : g * 128);
       // per-warp row sums of the epilogue live in the first row group (2 KB) of the group's P buffer: the last
       // PV of the segment has been waited for by then, and every tile rewrites that row group
       float* lsum_s = reinterpret_cast<float*>(sP + g * PBYTES);
-      float l_loc[NRP];
+      float l_loc[NR];
       uint32_t jt = 0;
       int seg = 0;
       bool ok = true;
@@ -471,19 +487,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const int item = (int)(f / Tt), tile0 = (int)(f - (long long)item * Tt);
         const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
         const int n = (int)(seg_end - f);
-        if (t < NRP) m_s[t] = kNegBig;
+        if (t < NR) m_s[r0 + t] = kNegBig;
 #pragma unroll
-        for (int i = 0; i < NRP; ++i) l_loc[i] = 0.f;
+        for (int i = 0; i < NR; ++i) l_loc[i] = 0.f;
         group_sync();
 
         bool aborted = false;
-        const int i_first = ((jt & 1) == (uint32_t)g) ? 0 : 1;      // this group's first tile in the segment
-        for (int i = i_first; i < n; i += 2) {
+        const int i_first = SC ? 0 : (((jt & 1) == (uint32_t)g) ? 0 : 1);      // this group's first tile in the segment
+        for (int i = i_first; i < n; i += (SC ? 1 : 2)) {
           const uint32_t j = jt + i, sb = j % NSB;
+          const uint32_t pb = SC ? (j & 1) : (uint32_t)g;            // P buffer of this tile
           const int tile = tile0 + i;
           const int rel = tile * kTile + t - a.n_ctx;                 // row r sees this key iff rel <= r
           const bool need_mask = (tile * kTile + kTile - 1 > a.n_ctx);
-          const uint32_t s_addr = tmem_S + lane_addr + sb * NRP;
+          const uint32_t s_addr = tmem_S + lane_addr + sb * NRP + r0;
           // A failed wait never leaves this loop on its own (the rest of the group would be left at a
           // named barrier): it clears `ok`, and the vote below takes all 128 threads out together.
           ok &= mbar_wait(bar(S_FULL + sb), (j / NSB) & 1, s_abort);
@@ -504,8 +521,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 if (lane == 0) {
 #pragma unroll
                   for (int e = 0; e < 16; ++e) {
-                    const bool masked = need_mask && rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16);
-                    if (!masked) m_s[c * 16 + e] = fmaf(__uint_as_float(raw[e]), a.scale_log2, 2.f * kRescaleThreshold);
+                    const bool masked = need_mask && rel > (int)(((uint32_t)(r0 + c * 16 + e) * a.g_magic) >> 16);
+                    if (!masked) m_s[r0 + c * 16 + e] = fmaf(__uint_as_float(raw[e]), a.scale_log2, 2.f * kRescaleThreshold);
                   }
                 }
                 __syncwarp();
@@ -522,7 +539,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               if (CW(c) == 16) tmem_ld16(s_addr + c * 16, xr[c]); else tmem_ld8_lo(s_addr + c * 16, xr[c]);
             tmem_wait_ld();
             float xm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            const float4* m4 = reinterpret_cast<const float4*>(m_s);
+            const float4* m4 = reinterpret_cast<const float4*>(m_s + r0);
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
               {
@@ -555,7 +572,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
                   for (int e = 0; e < CW(c); ++e) {
                     {
-                      if (rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16)) xr[c][e] = __float_as_uint(-INFINITY);
+                      if (rel > (int)(((uint32_t)(r0 + c * 16 + e) * a.g_magic) >> 16)) xr[c][e] = __float_as_uint(-INFINITY);
                       xmax = fmaxf(xmax, __uint_as_float(xr[c][e]));
                     }
                   }
@@ -584,43 +601,46 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
               for (int e = 0; e < 16; ++e) {
                 float v = __uint_as_float(raw[e]) * a.scale_log2;
-                if (e >= cw || (need_mask && rel > (int)(((uint32_t)(c * 16 + e) * a.g_magic) >> 16))) v = -INFINITY;
+                if (e >= cw || (need_mask && rel > (int)(((uint32_t)(r0 + c * 16 + e) * a.g_magic) >> 16))) v = -INFINITY;
                 // warp maximum in one instruction on the order-preserving integer image of the float
                 const int ov = __reduce_max_sync(0xffffffffu, f2ord(v));
-                if (lane == 0 && e < cw) atomicMax(&newmax_s[c * 16 + e], ov);
+                if (lane == 0 && e < cw) atomicMax(&newmax_s[r0 + c * 16 + e], ov);
               }
             }
             group_sync();
-            if (t < NRP) {
-              const float mo = m_s[t], mn = fmaxf(mo, ord2f(newmax_s[t]));
-              fac_s[t] = ex2(mo - mn);                 // 0 when the row had seen nothing, 1 when nothing changed
-              m_s[t] = mn;
-              newmax_s[t] = f2ord(-INFINITY);
+            if (t < NR) {
+              const int row = r0 + t;
+              const float mo = m_s[row], mn = fmaxf(mo, ord2f(newmax_s[row]));
+              fac_s[row] = ex2(mo - mn);               // 0 when the row had seen nothing, 1 when nothing changed
+              m_s[row] = mn;
+              newmax_s[row] = f2ord(-INFINITY);
             }
             group_sync();
 #pragma unroll
-            for (int k = 0; k < NRP; ++k) l_loc[k] *= fac_s[k];
-            if (i >= 2) {
-              // the accumulator holds this group's earlier tiles: wait until the last of them has been added
-              ok &= mbar_wait(bar(P_FREE + g), ((j >> 1) - 1) & 1, s_abort);
+            for (int k = 0; k < NR; ++k) l_loc[k] *= fac_s[r0 + k];
+            if (i >= (SC ? 1 : 2)) {
+              // the accumulator holds earlier tiles of the segment: wait until the last of them has been added
+              // (split-column mode: the tile before this one, whose P buffer is the other one)
+              const uint32_t jp = SC ? j - 1 : j - 2;
+              ok &= mbar_wait(bar(P_FREE + (SC ? (jp & 1) : (uint32_t)g)), (jp >> 1) & 1, s_abort);
               tc_fence_after();
 #pragma unroll 1
               for (int c = 0; c < NCH; ++c) {
                 uint32_t o[16];
-                tmem_ld16(tmem_O + lane_addr + g * NRP + c * 16, o);
+                tmem_ld16(tmem_O + lane_addr + (SC ? 0 : g * NRP) + r0 + c * 16, o);
                 tmem_wait_ld();
                 reg_fence16(o);
 #pragma unroll
-                for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * fac_s[c * 16 + e]);
-                tmem_st16(tmem_O + lane_addr + g * NRP + c * 16, o);
+                for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * fac_s[r0 + c * 16 + e]);
+                tmem_st16(tmem_O + lane_addr + (SC ? 0 : g * NRP) + r0 + c * 16, o);
               }
               tmem_wait_st();
             }
           }
           if (aborted) break;
           // ---- probabilities, running sums, bf16 P in the MN-major core-matrix layout ----
-          if (i >= 2) ok &= mbar_wait(bar(P_FREE + g), ((j >> 1) - 1) & 1, s_abort);
-          unsigned char* pdst = sP + g * PBYTES + t * 16;
+          if (i >= 2) ok &= mbar_wait(bar(P_FREE + pb), ((j >> 1) - 1) & 1, s_abort);     // the buffer's last reader: tile j - 2
+          unsigned char* pdst = sP + pb * PBYTES + (r0 >> 3) * 2048 + t * 16;
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
             {
@@ -651,35 +671,40 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         ok &= mbar_wait(bar(O_FULL), seg & 1, s_abort);
         tc_fence_after();
         if (seg_end < f_end) q_store();
-        const long long slot = ((long long)blockIdx.x * a.seg_max + (item - item_first)) * 2 + g;
+        // (split-column mode: both groups fill the segment's first slot, each its own rows; the second slot is marked empty)
+        const long long slot = ((long long)blockIdx.x * a.seg_max + (item - item_first)) * 2 + (SC ? 0 : g);
         float* po = a.part_o + slot * NRP * 128;
         const bool has_tiles = i_first < n;
         if (has_tiles) {
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
             uint32_t o[16];
-            tmem_ld16(tmem_O + lane_addr + g * NRP + c * 16, o);
+            tmem_ld16(tmem_O + lane_addr + (SC ? 0 : g * NRP) + r0 + c * 16, o);
             tmem_wait_ld();
             reg_fence16(o);
 #pragma unroll
-            for (int e = 0; e < 16; ++e) po[(long long)(c * 16 + e) * 128 + t] = __uint_as_float(o[e]);
+            for (int e = 0; e < 16; ++e) po[(long long)(r0 + c * 16 + e) * 128 + t] = __uint_as_float(o[e]);
           }
         }
         tc_fence_before();
         mbar_arrive(bar(O_FREE));
 #pragma unroll
-        for (int k = 0; k < NRP; ++k) {
+        for (int k = 0; k < NR; ++k) {
           float v = l_loc[k];
 #pragma unroll
           for (int sh = 16; sh >= 1; sh >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sh);
           if (lane == 0) lsum_s[q4 * 128 + k] = v;
         }
         group_sync();
-        if (t < NRP) {
+        if (t < NR) {
           const float* ls = lsum_s;
           const float l = ((ls[t] + ls[128 + t]) + ls[256 + t]) + ls[384 + t];
-          a.part_ml[(slot * NRP + t) * 2] = has_tiles ? m_s[t] : kNegBig;
-          a.part_ml[(slot * NRP + t) * 2 + 1] = has_tiles ? l : 0.f;
+          a.part_ml[(slot * NRP + r0 + t) * 2] = has_tiles ? m_s[r0 + t] : kNegBig;
+          a.part_ml[(slot * NRP + r0 + t) * 2 + 1] = has_tiles ? l : 0.f;
+        }
+        if (SC && g == 1 && t < NRP) {           // the slot of the segment that nobody fills: "saw no key"
+          a.part_ml[((slot + 1) * NRP + t) * 2] = kNegBig;
+          a.part_ml[((slot + 1) * NRP + t) * 2 + 1] = 0.f;
         }
         group_sync();
         jt += n;
@@ -932,7 +957,7 @@ __global__ void __launch_bounds__(128) attn_tc_combine_many_kernel(const Combine
 // lse of every row known, a thread turns its key's scores into probabilities and adds them over the
 // query rows, which in this orientation is a thread-local sum: mass_part[kv head][key].
 // ---------------------------------------------------------------------------------------------
-constexpr int kMassKStages = 4;
+constexpr int kMassKStages = 6;             // K tiles in flight: the kernel holds no V, P or accumulators, so shared memory allows six
 
 struct TcMassArgs {
   const __nv_bfloat16* q;
@@ -953,7 +978,8 @@ struct TcMassArgs {
 template <int NRP>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a) {
-  constexpr int NCH = NRP / 16;
+  constexpr bool SC = split_cols(NRP);     // both groups on every tile, half of the query-row columns each (two partial sums per key)
+  constexpr int NCH = SC ? NRP / 32 : NRP / 16;
   constexpr int QBOX = NRP * 128;
   constexpr int NSB = (512 / NRP) >= 4 ? 4 : (512 / NRP);
   constexpr uint32_t NEED = NSB * NRP;
@@ -968,7 +994,8 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
   uint64_t* bars = reinterpret_cast<uint64_t*>(s_lse + 128);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 24);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-  enum { K_FULL = 0, K_EMPTY = 4, S_FULL = 8, S_FREE = 12, Q_READY = 16 };
+  enum { K_FULL = 0, K_EMPTY = kMassKStages, S_FULL = 2 * kMassKStages, S_FREE = 2 * kMassKStages + 4, Q_READY = 2 * kMassKStages + 8 };
+  static_assert(2 * kMassKStages + 9 <= 24, "barrier storage");
   auto bar = [&](int i) { return smem_addr(bars + i); };
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const long long W = a.total_tiles;
@@ -976,10 +1003,8 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
   const int Tt = a.tiles_per_item;
 
   if (tid == 0) {
-    for (int i = 0; i < 4; ++i) {
-      mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1);
-      mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), kGroupThreads);
-    }
+    for (int i = 0; i < kMassKStages; ++i) { mbar_init(bar(K_FULL + i), 1); mbar_init(bar(K_EMPTY + i), 1); }
+    for (int i = 0; i < 4; ++i) { mbar_init(bar(S_FULL + i), 1); mbar_init(bar(S_FREE + i), SC ? kSoftmaxThreads : kGroupThreads); }
     mbar_init(bar(Q_READY), kSoftmaxThreads);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1045,7 +1070,8 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
       const int q4 = warp & 3, g = (warp - 4) >> 2;
       const int t = q4 * 32 + lane, st = tid - 128;
       const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
-      const int nch_valid = (a.rows + 15) >> 4;
+      const int r0 = SC ? g * (NCH * 16) : 0;                    // first query-row column of this thread's share
+      const int nch_valid = min(NCH, max(0, (a.rows - r0 + 15) >> 4));
       uint32_t jt = 0;
       int seg = 0;
       bool ok = true;
@@ -1090,9 +1116,9 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
           mbar_arrive(bar(Q_READY));
         }
         softmax_bar_or(false);                     // s_lse visible to both groups
-        const int i_first = ((jt & 1) == (uint32_t)g) ? 0 : 1;
-        float* out = a.part_mass + ((long long)zrow * a.Hkv + kvh) * a.T_pad;
-        for (int i = i_first; i < n; i += 2) {
+        const int i_first = SC ? 0 : (((jt & 1) == (uint32_t)g) ? 0 : 1);
+        float* out = a.part_mass + (((long long)zrow * a.Hkv + kvh) * (SC ? 2 : 1) + (SC ? g : 0)) * a.T_pad;
+        for (int i = i_first; i < n; i += (SC ? 1 : 2)) {
           const uint32_t j = jt + i, sb = j % NSB;
           const int tile = tile0 + i;
           const int key = tile * kTile + t;
@@ -1100,7 +1126,7 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
           const bool need_mask = (tile * kTile + kTile - 1 > a.n_ctx);
           ok &= mbar_wait(bar(S_FULL + sb), (j / NSB) & 1, s_abort);
           tc_fence_after();
-          const uint32_t s_addr = tmem + lane_addr + sb * NRP;
+          const uint32_t s_addr = tmem + lane_addr + sb * NRP + r0;
           uint32_t xr[NCH][16];
 #pragma unroll
           for (int c = 0; c < NCH; ++c)
@@ -1109,7 +1135,7 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
           tc_fence_before();
           mbar_arrive(bar(S_FREE + sb));
           float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          const float4* l4 = reinterpret_cast<const float4*>(s_lse);
+          const float4* l4 = reinterpret_cast<const float4*>(s_lse + r0);
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
             if (c < nch_valid) {
@@ -1122,7 +1148,7 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
                 float x2 = fmaf(__uint_as_float(xr[c][4 * q + 2]), a.scale_log2, -lq.z);
                 float x3 = fmaf(__uint_as_float(xr[c][4 * q + 3]), a.scale_log2, -lq.w);
                 if (need_mask) {
-                  const int n0 = c * 16 + 4 * q;
+                  const int n0 = r0 + c * 16 + 4 * q;
                   if (rel > (int)(((uint32_t)(n0 + 0) * a.g_magic) >> 16)) x0 = -INFINITY;
                   if (rel > (int)(((uint32_t)(n0 + 1) * a.g_magic) >> 16)) x1 = -INFINITY;
                   if (rel > (int)(((uint32_t)(n0 + 2) * a.g_magic) >> 16)) x2 = -INFINITY;
@@ -1157,6 +1183,7 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
   }
 }
 
+// part: [n_mass][n_part][T_pad] with n_part = KV heads (x 2 in split-column mode), summed in fixed order
 __global__ void mass_reduce_tc_kernel(const float* part, float* mass, int Hkv, int T, int T_pad, long long mass_ls) {
   pdl_launch_dependents();
   pdl_wait();
@@ -1207,10 +1234,14 @@ constexpr int tc_smem_bytes() {
 template <int NRP>
 void launch_tc(const CUtensorMap& mk, const CUtensorMap& mv, const TcArgs& a, cudaStream_t s) {
   constexpr int smem = tc_smem_bytes<NRP>();
-  if (a.rows <= NRP - 8) {
-    cudaFuncSetAttribute(attn_tc_kernel<NRP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    attn_tc_kernel<NRP, true><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
-  } else {
+  if constexpr (!split_cols(NRP)) {
+    if (a.rows <= NRP - 8) {
+      cudaFuncSetAttribute(attn_tc_kernel<NRP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      attn_tc_kernel<NRP, true><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
+      return;
+    }
+  }
+  {
     cudaFuncSetAttribute(attn_tc_kernel<NRP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     attn_tc_kernel<NRP, false><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
   }
@@ -1258,7 +1289,8 @@ pvlm_status launch_attn_mass_tc(const pvlm_attn_params& p, const float* lse2, fl
     default: return PVLM_ERR_UNSUPPORTED;
   }
   const cudaError_t e = launch_dependent(mass_reduce_tc_kernel, dim3(ceil_div(T, 256), n_mass), dim3(256), 0, s,
-                                         (const float*)part_mass, p.mass, p.Hkv, T, a.T_pad, p.mass_layer_stride);
+                                         (const float*)part_mass, p.mass, p.Hkv * (split_cols(nrp) ? 2 : 1), T, a.T_pad,
+                                         p.mass_layer_stride);
   if (e != cudaSuccess) set_cuda_error((int)e);
   return check_launch();
 }
@@ -1305,8 +1337,7 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   a.tiles_per_item = plan.tiles_per_item; a.total_tiles = plan.total_tiles; a.seg_max = plan.seg_max; a.n_cta = plan.n_cta;
   a.g_magic = (65536u + a.G - 1) / a.G;
   {
-    const int nsb = (512 - 2 * plan.nrp) / plan.nrp >= 4 ? 4 : (512 - 2 * plan.nrp) / plan.nrp;
-    a.lookahead = nsb - 1;
+    a.lookahead = s_bufs(plan.nrp) - 1;
   }
   cudaMemsetAsync(a.status, 0, 4, s);
   if (p.prof_event_begin) cudaEventRecord((cudaEvent_t)p.prof_event_begin, s);
