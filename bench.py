@@ -667,8 +667,10 @@ def decode_pipeline_leg(cfg, dev, torch, binding, Q, K, V, O, args):
     ur = torch.rand((n_tok,), generator=g, device=dev)
     ws = [torch.empty(256 << 20, dtype=torch.uint8, device=dev) for _ in range(2)]
 
+    O_dec = torch.empty_like(O)                        # its own output: the step's O is compared with the oracle later
+
     def blocks(t_ctas, d_ctas):
-        pt = binding.attn_params(Q, K[:, :n0 + cfg.R], V[:, :n0 + cfg.R], n0, O, None, None, workspace=ws[0], max_ctas=t_ctas)
+        pt = binding.attn_params(Q, K[:, :n0 + cfg.R], V[:, :n0 + cfg.R], n0, O_dec, None, None, workspace=ws[0], max_ctas=t_ctas)
         pd = binding.attn_params(Qd, Kd[:, :S2 + 1], Vd[:, :S2 + 1], S2, Od, None, None, workspace=ws[1], max_ctas=d_ctas)
         return pt, pd
 

@@ -69,6 +69,7 @@ struct TcArgs {
   int n_cta;
   uint32_t g_magic;          // ceil(2^16 / G): row / G == (row * g_magic) >> 16 for row < 128
   int lookahead;             // score tiles the issuer keeps in flight past the tile whose PV it issues next
+  int l2_hints;              // 1: a mass pass over the same layers follows: K is asked to stay in L2, V to leave first
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -165,6 +166,24 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
+}
+// The same load with an L2 eviction-priority hint (a policy word made by l2_policy_*).
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 // One lane of a converged warp (the same lane every time).
 __device__ __forceinline__ bool elect_one() {
@@ -309,6 +328,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         uint32_t u = 0;                          // loads issued so far (ring position)
         uint32_t jt = 0;
         bool ok = true;
+        // K tiles of a call whose mass pass re-reads them are asked to stay in L2, V tiles (read once) to leave first
+        const uint64_t pol_k = l2_policy_evict_last(), pol_v = l2_policy_evict_first();
         auto load = [&](const CUtensorMap* map, uint32_t full_bar, long long f) -> bool {
           const uint32_t slot = u % NS;
           if (u >= NS && !mbar_wait(bar(EMPTY + slot), ((u / NS) - 1) & 1, s_abort)) return false;
@@ -316,8 +337,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
           const uint32_t dst = smem_addr(sRing + slot * kTileBytes);
           mbar_expect_tx(full_bar, kTileBytes);
-          tma_load_4d(dst, map, full_bar, 0, kvh, tile * kTile, layer);
-          tma_load_4d(dst + kBoxBytes, map, full_bar, 64, kvh, tile * kTile, layer);
+          if (a.l2_hints) {
+            const uint64_t pol = map == &tm_k ? pol_k : pol_v;
+            tma_load_4d_hint(dst, map, full_bar, 0, kvh, tile * kTile, layer, pol);
+            tma_load_4d_hint(dst + kBoxBytes, map, full_bar, 64, kvh, tile * kTile, layer, pol);
+          } else {
+            tma_load_4d(dst, map, full_bar, 0, kvh, tile * kTile, layer);
+            tma_load_4d(dst + kBoxBytes, map, full_bar, 64, kvh, tile * kTile, layer);
+          }
           ++u;
           return true;
         };
@@ -1024,8 +1051,10 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
     const uint32_t total = (uint32_t)(f_end - f_begin);
     if (warp == 0) {
       if (lane == 0) {
+        // A CTA walks its tile range BACKWARDS: when this pass covers the same layers as the main pass (a one-layer
+        // call) its range is the one that CTA streamed there, and the tiles it read last are the likeliest to be in L2 still.
         for (uint32_t j = 0; j < total; ++j) {
-          const long long f = f_begin + j;
+          const long long f = f_end - 1 - j;
           const int item = (int)(f / Tt), tile = (int)(f - (long long)item * Tt);
           const int zrow = item / a.Hkv, kvh = item - zrow * a.Hkv;
           const int layer = a.mass_listed ? a.mass_layer[zrow] : zrow;
@@ -1042,10 +1071,10 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
         uint32_t jt = 0;
         int seg = 0;
         bool ok = true;
-        for (long long f = f_begin; f < f_end && ok; ++seg) {
-          const int item = (int)(f / Tt);
-          const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
-          const int n = (int)(seg_end - f);
+        for (long long fh = f_end - 1; fh >= f_begin && ok; ++seg) {        // fh: the segment's highest tile, processed first
+          const int item = (int)(fh / Tt);
+          const long long seg_lo = max(f_begin, (long long)item * Tt);
+          const int n = (int)(fh - seg_lo + 1);
           if (!mbar_wait(bar(Q_READY), seg & 1, s_abort)) break;
           tc_fence_after();
           for (int i = 0; i < n; ++i) {
@@ -1063,7 +1092,7 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
             tc_commit(bar(K_EMPTY + ks));
           }
           jt += n;
-          f = seg_end;
+          fh = seg_lo - 1;
         }
       }
     } else if (warp >= 4) {
@@ -1075,10 +1104,10 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
       uint32_t jt = 0;
       int seg = 0;
       bool ok = true;
-      for (long long f = f_begin; f < f_end; ++seg) {
-        const int item = (int)(f / Tt), tile0 = (int)(f - (long long)item * Tt);
-        const long long seg_end = min(f_end, (long long)(item + 1) * Tt);
-        const int n = (int)(seg_end - f);
+      for (long long fh = f_end - 1; fh >= f_begin; ++seg) {
+        const int item = (int)(fh / Tt), tile_hi = (int)(fh - (long long)item * Tt);
+        const long long seg_lo = max(f_begin, (long long)item * Tt);
+        const int n = (int)(fh - seg_lo + 1);
         const int zrow = item / a.Hkv, kvh = item - zrow * a.Hkv;
         const int layer = a.mass_listed ? a.mass_layer[zrow] : zrow;
         {
@@ -1120,7 +1149,7 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
         float* out = a.part_mass + (((long long)zrow * a.Hkv + kvh) * (SC ? 2 : 1) + (SC ? g : 0)) * a.T_pad;
         for (int i = i_first; i < n; i += (SC ? 1 : 2)) {
           const uint32_t j = jt + i, sb = j % NSB;
-          const int tile = tile0 + i;
+          const int tile = tile_hi - i;
           const int key = tile * kTile + t;
           const int rel = key - a.n_ctx;
           const bool need_mask = (tile * kTile + kTile - 1 > a.n_ctx);
@@ -1166,7 +1195,7 @@ attn_tc_mass_kernel(const __grid_constant__ CUtensorMap tm_k, const TcMassArgs a
         // all score MMAs of the segment have been consumed by one of the groups: Q may be replaced
         if (softmax_bar_or(!ok)) break;
         jt += n;
-        f = seg_end;
+        fh = seg_lo - 1;
       }
     }
   }
@@ -1338,6 +1367,8 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   a.g_magic = (65536u + a.G - 1) / a.G;
   {
     a.lookahead = s_bufs(plan.nrp) - 1;
+    // worth it only where the mass pass re-reads a sizeable share of what this launch streams: every layer's mass wanted
+    a.l2_hints = (p.mass != nullptr && (p.mass_layers == nullptr || p.n_mass_layers == p.n_layers)) ? 1 : 0;
   }
   cudaMemsetAsync(a.status, 0, 4, s);
   if (p.prof_event_begin) cudaEventRecord((cudaEvent_t)p.prof_event_begin, s);
