@@ -799,20 +799,28 @@ __global__ void __launch_bounds__(128) attn_tc_combine_kernel(const CombineArgs 
     // few partials per item (long tile runs): a warp merges whole rows on its own, no block barriers
     const int layer = item / a.Hkv, kvh = item - layer * a.Hkv;
     for (int row = blockIdx.y * 4 + warp; row < a.rows; row += 4 * gridDim.y) {
+      // all (m, l) pairs first, then every partial's row piece in flight at once, then a fixed-order sum
+      float2 ml[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        ml[i] = i < n ? *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2) : make_float2(kNegBig, 0.f);
       float mstar = -INFINITY;
-      for (int i = 0; i < n; ++i) {
-        const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
-        if (ml.y > 0.f) mstar = fmaxf(mstar, ml.x);
-      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (ml[i].y > 0.f) mstar = fmaxf(mstar, ml[i].x);
+      float4 o[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        o[i] = (i < n && ml[i].y > 0.f) ? *reinterpret_cast<const float4*>(a.part_o + (s_slot[i] * a.nrp + row) * 128 + lane * 4)
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
       float l = 0.f;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int i = 0; i < n; ++i) {
-        const float2 ml = *reinterpret_cast<const float2*>(a.part_ml + (s_slot[i] * a.nrp + row) * 2);
-        if (!(ml.y > 0.f)) continue;
-        const float w = ex2(ml.x - mstar);
-        l += ml.y * w;
-        const float4 o = *reinterpret_cast<const float4*>(a.part_o + (s_slot[i] * a.nrp + row) * 128 + lane * 4);
-        acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (!(i < n && ml[i].y > 0.f)) continue;
+        const float w = ex2(ml[i].x - mstar);
+        l += ml[i].y * w;
+        acc.x += o[i].x * w; acc.y += o[i].y * w; acc.z += o[i].z * w; acc.w += o[i].w * w;
       }
       const float inv = 1.f / l;
       const int r = row / a.G, g = row - r * a.G;
