@@ -10,6 +10,10 @@ namespace pvlm {
 namespace {
 
 constexpr int kSelThreads = 1024;
+#ifndef PVLM_WIDE_SELECT_MIN
+#define PVLM_WIDE_SELECT_MIN 32769
+#endif
+constexpr int kWideSelectMinTokens = PVLM_WIDE_SELECT_MIN;   // from this many tokens on the selection uses a 16-CTA cluster
 constexpr int kSelWarps = kSelThreads / 32;
 
 // Order-preserving map fp32 -> uint32 (larger float => larger key); -0.0 maps
@@ -246,16 +250,16 @@ __global__ void __launch_bounds__(kSelThreads) uvprune_select_reg_kernel(const S
 // adds up all eight histograms through distributed shared memory, so all CTAs derive the same
 // threshold without any global-memory round trip.  The ordered compaction needs one more exchange
 // (per-CTA counts of greater and of equal keys).  m <= 8 * 1024 * ITEMS.
-constexpr int kSelCluster = 8;
-
-template <int ITEMS>
+// kSelCluster: CTAs per cluster, 8 (portable) or 16 (needs the non-portable cluster size attribute at launch).
+template <int ITEMS, int kSelCluster>
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 uvprune_select_cluster_kernel(const SelArgs a) {
   pdl_wait();                  // the masses may come from the kernel right before (programmatic dependent launch)
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   const unsigned rank = cluster.block_rank();
-  __shared__ unsigned int hist[256];                     // this CTA's histogram of the pass (read remotely)
+  __shared__ unsigned int hist[2][256];                  // this CTA's histogram of the pass (read remotely); two buffers, so
+                                                         // that one cluster barrier per pass is enough (see below)
   __shared__ unsigned int hist_l[256 * 32];
   __shared__ unsigned int s_prefix, s_remaining;
   __shared__ int s_cnt[2];                               // (greater, equal) counts of this CTA (read remotely)
@@ -278,7 +282,9 @@ uvprune_select_cluster_kernel(const SelArgs a) {
   if (a.k == 0) return;                                  // uniform over the cluster: nobody reaches a cluster barrier
   if (tid == 0) { s_prefix = 0u; s_remaining = (unsigned)a.k; }
   uint32_t mask = 0u;
-  for (int shift = 24; shift >= 0; shift -= 8) {
+  int pass = 0;
+  for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
+    unsigned int* hist_p = hist[pass & 1];
     for (int i = tid; i < 256 * 32; i += kSelThreads) hist_l[i] = 0u;
     __syncthreads();
     const uint32_t prefix = s_prefix;
@@ -291,13 +297,16 @@ uvprune_select_cluster_kernel(const SelArgs a) {
       unsigned t = 0;
 #pragma unroll 8
       for (int j = 0; j < 32; ++j) t += hist_l[(tid << 5) + ((j + tid) & 31)];
-      hist[tid] = t;
+      hist_p[tid] = t;
     }
-    cluster.sync();                                      // all eight histograms are complete
+    // Every CTA's histogram of this pass is complete.  No second barrier after the remote reads: the next pass writes the
+    // OTHER buffer, and this one is written again two passes on, behind the next pass's barrier, which a CTA reaches only
+    // after its reads here.
+    cluster.sync();
     unsigned v = 0, incl = 0;
     if (tid < 256) {
 #pragma unroll
-      for (int r = 0; r < kSelCluster; ++r) v += cluster.map_shared_rank(hist, r)[255 - tid];   // descending digit order
+      for (int r = 0; r < kSelCluster; ++r) v += cluster.map_shared_rank(hist_p, r)[255 - tid];   // descending digit order
       incl = v;
 #pragma unroll
       for (int sh = 1; sh < 32; sh <<= 1) {
@@ -316,7 +325,7 @@ uvprune_select_cluster_kernel(const SelArgs a) {
       }
     }
     mask |= (0xFFu << shift);
-    cluster.sync();                                      // remote reads of `hist` are done; s_prefix is visible
+    __syncthreads();                                     // s_prefix / s_remaining are visible to the whole CTA
   }
   const uint32_t tau = s_prefix;
   const int take_eq = (int)s_remaining;
@@ -425,11 +434,20 @@ pvlm_status launch_uvprune_parts(const pvlm_prune_params& p, bool select, int pa
   sa.k = p.k;
   if (select && p.m > 0) {
     const bool one_cta = option_value(PVLM_OPT_SELECT_ONE_CTA) != 0;    // single-CTA kernels only: the tests' second implementation
-    const dim3 cl(kSelCluster), one(1), th(kSelThreads);
+    const dim3 cl8(8), cl16(16), one(1), th(kSelThreads);
     cudaError_t e;
-    if (!one_cta && p.m <= kSelCluster * kSelThreads * 4) e = launch_dependent(uvprune_select_cluster_kernel<4>, cl, th, 0, s, sa);
-    else if (!one_cta && p.m <= kSelCluster * kSelThreads * 16) e = launch_dependent(uvprune_select_cluster_kernel<16>, cl, th, 0, s, sa);
-    else if (!one_cta && p.m <= kSelCluster * kSelThreads * 32) e = launch_dependent(uvprune_select_cluster_kernel<32>, cl, th, 0, s, sa);
+    // larger token counts go to a 16-CTA cluster (half the keys per thread); that size is not portable, so the kernels are
+    // told once that it is allowed here
+    static const bool wide_ok = [] {
+      return cudaFuncSetAttribute(uvprune_select_cluster_kernel<8, 16>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+             cudaFuncSetAttribute(uvprune_select_cluster_kernel<16, 16>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+    }();
+    const int wide_min = kWideSelectMinTokens;
+    if (!one_cta && p.m <= 8 * kSelThreads * 4 && p.m < wide_min) e = launch_dependent(uvprune_select_cluster_kernel<4, 8>, cl8, th, 0, s, sa);
+    else if (!one_cta && wide_ok && p.m <= 16 * kSelThreads * 8) e = launch_dependent(uvprune_select_cluster_kernel<8, 16>, cl16, th, 0, s, sa);
+    else if (!one_cta && wide_ok && p.m <= 16 * kSelThreads * 16) e = launch_dependent(uvprune_select_cluster_kernel<16, 16>, cl16, th, 0, s, sa);
+    else if (!one_cta && p.m <= 8 * kSelThreads * 16) e = launch_dependent(uvprune_select_cluster_kernel<16, 8>, cl8, th, 0, s, sa);
+    else if (!one_cta && p.m <= 8 * kSelThreads * 32) e = launch_dependent(uvprune_select_cluster_kernel<32, 8>, cl8, th, 0, s, sa);
     else if (p.m <= 32 * kSelThreads) e = launch_dependent(uvprune_select_reg_kernel<32>, one, th, 0, s, sa);
     else e = launch_dependent(uvprune_select_kernel, one, th, 0, s, sa);
     if (e != cudaSuccess) set_cuda_error((int)e);

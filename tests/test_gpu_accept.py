@@ -119,7 +119,10 @@ def test_full_vocab_configs(cid):
         check_against_oracle(tl, dl, tok, u)
 
 
-@pytest.mark.parametrize("V,gamma", [(1, 1), (2, 3), (3, 1), (5, 2), (16, 4), (17, 64), (1023, 5), (1025, 7), (4097, 2)])
+@pytest.mark.parametrize("V,gamma", [(1, 1), (2, 3), (3, 1), (5, 2), (16, 4), (17, 64), (1023, 5), (1025, 7), (4097, 2),
+                                     # around the sizes at which the tail team grows to 2, 4 and 8 CTAs, and a vocabulary whose
+                                     # warp ranges are longer than the steps kept in registers (the recomputing walk)
+                                     (20480, 3), (20481, 3), (40961, 2), (81921, 2), (200003, 1), (600001, 1)])
 def test_small_and_ragged_vocab(V, gamma):
     rng = np.random.default_rng(V * 100 + gamma)
     for trial in range(4):
