@@ -435,21 +435,29 @@ pvlm_status launch_uvprune_parts(const pvlm_prune_params& p, bool select, int pa
   if (select && p.m > 0) {
     const bool one_cta = option_value(PVLM_OPT_SELECT_ONE_CTA) != 0;    // single-CTA kernels only: the tests' second implementation
     const dim3 cl8(8), cl16(16), one(1), th(kSelThreads);
-    cudaError_t e;
-    // larger token counts go to a 16-CTA cluster (half the keys per thread); that size is not portable, so the kernels are
-    // told once that it is allowed here
-    static const bool wide_ok = [] {
-      return cudaFuncSetAttribute(uvprune_select_cluster_kernel<8, 16>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
-             cudaFuncSetAttribute(uvprune_select_cluster_kernel<16, 16>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
-    }();
-    const int wide_min = kWideSelectMinTokens;
-    if (!one_cta && p.m <= 8 * kSelThreads * 4 && p.m < wide_min) e = launch_dependent(uvprune_select_cluster_kernel<4, 8>, cl8, th, 0, s, sa);
-    else if (!one_cta && wide_ok && p.m <= 16 * kSelThreads * 8) e = launch_dependent(uvprune_select_cluster_kernel<8, 16>, cl16, th, 0, s, sa);
-    else if (!one_cta && wide_ok && p.m <= 16 * kSelThreads * 16) e = launch_dependent(uvprune_select_cluster_kernel<16, 16>, cl16, th, 0, s, sa);
-    else if (!one_cta && p.m <= 8 * kSelThreads * 16) e = launch_dependent(uvprune_select_cluster_kernel<16, 8>, cl8, th, 0, s, sa);
-    else if (!one_cta && p.m <= 8 * kSelThreads * 32) e = launch_dependent(uvprune_select_cluster_kernel<32, 8>, cl8, th, 0, s, sa);
-    else if (p.m <= 32 * kSelThreads) e = launch_dependent(uvprune_select_reg_kernel<32>, one, th, 0, s, sa);
-    else e = launch_dependent(uvprune_select_kernel, one, th, 0, s, sa);
+    cudaError_t e = cudaErrorUnknown;
+    bool launched = false;
+    // Larger token counts go to a 16-CTA cluster (half the keys per thread).  That size is not portable, so the kernel is
+    // told that it is allowed: a per-device function attribute, hence set with the launch, not once per process.
+    if (!one_cta && p.m >= kWideSelectMinTokens && p.m <= 16 * kSelThreads * 16) {
+      auto wide = [&](auto kernel) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+          (void)cudaGetLastError();
+          return;                                           // this device will not have it: the 8-CTA kernels below
+        }
+        e = launch_dependent(kernel, cl16, th, 0, s, sa);
+        launched = true;
+      };
+      if (p.m <= 16 * kSelThreads * 8) wide(uvprune_select_cluster_kernel<8, 16>);
+      else wide(uvprune_select_cluster_kernel<16, 16>);
+    }
+    if (!launched) {
+      if (!one_cta && p.m <= 8 * kSelThreads * 4) e = launch_dependent(uvprune_select_cluster_kernel<4, 8>, cl8, th, 0, s, sa);
+      else if (!one_cta && p.m <= 8 * kSelThreads * 16) e = launch_dependent(uvprune_select_cluster_kernel<16, 8>, cl8, th, 0, s, sa);
+      else if (!one_cta && p.m <= 8 * kSelThreads * 32) e = launch_dependent(uvprune_select_cluster_kernel<32, 8>, cl8, th, 0, s, sa);
+      else if (p.m <= 32 * kSelThreads) e = launch_dependent(uvprune_select_reg_kernel<32>, one, th, 0, s, sa);
+      else e = launch_dependent(uvprune_select_kernel, one, th, 0, s, sa);
+    }
     if (e != cudaSuccess) set_cuda_error((int)e);
   }
   if (p.src_k && part != 3) {

@@ -188,9 +188,11 @@ def test_mma_sync_path_still_matches(pvlm_option):
         run_case(qb, kb, vb, n_ctx)
 
 
-@pytest.mark.parametrize("Hq,Hkv,R", [(16, 2, 13), (16, 2, 16), (14, 2, 15)])
+@pytest.mark.parametrize("Hq,Hkv,R", [(16, 2, 13), (16, 2, 16), (14, 2, 15), (16, 2, 11), (16, 2, 12), (14, 2, 12)])
 def test_wide_row_groups_on_the_tensor_core_path(Hq, Hkv, R, pvlm_option):
-    """97..128 query rows per KV head (3 ring slots, 2 score buffers): long tile runs with several segments per CTA."""
+    """81..128 query rows per KV head: 96 and 128 padded rows run in split-column mode (both softmax groups on every tile,
+    half of the rows each; 84, 88, 96 and 128 rows here), 112 padded rows (104, 105 rows) on alternate tiles with 3 ring
+    slots and 2 score buffers.  Long tile runs with several segments per CTA."""
     pvlm_option("attn_max_ctas", 3)
     n_ctx = 2100
     qb, kb, vb = wl.make_qkv(Hq, Hkv, 128, R, n_ctx + R, sink=True, seed=500 + R)
