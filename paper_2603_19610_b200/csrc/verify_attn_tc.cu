@@ -1401,7 +1401,8 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
   c.D = p.D;
   {
     const int items = p.Hkv * p.n_layers;
-    int rows_y = 2048 / items;                            // enough blocks to fill the GPU, not tens of thousands
+    int rows_y = 2048 / items;                            // enough blocks to fill the GPU, not tens of thousands (1024 / 4096 / 8192
+                                                          // blocks measured 23.7 / 26.8 / 31.7 us against 24.9 at the 64-layer config)
     rows_y = rows_y < 1 ? 1 : (rows_y > a.rows ? a.rows : rows_y);
     // an item's tiles are spread over at most this many CTAs, each with two partials
     const long long ctas_per_item = ((long long)plan.tiles_per_item * plan.n_cta + plan.total_tiles - 1) / plan.total_tiles + 1;
