@@ -187,16 +187,24 @@ pvlm_status pvlm_uvprune_select_gather(const pvlm_prune_params *p, void *stream)
  * hidden: bf16 [rows][d] token representations of one layer, row stride
  * hidden_row_stride elements; visual rows [vis_start, vis_start+m), text
  * rows [text_start, text_start+n).
- * Supported: d % 8 == 0, 8 <= d <= 16384; hidden 16-byte aligned, row stride
- * a multiple of 8; m >= 0, n >= 0.
+ * n_layers > 1 computes that many layers in one call (the two end layers of
+ * Eq. 2 normally): layer l's hidden states start hidden_layer_stride elements
+ * after layer l-1's and its result goes to sim + l * sim_layer_stride; each
+ * kernel then covers all layers in one launch.  n_layers <= 1 is one layer
+ * and the two layer strides are ignored.
+ * Supported: d % 8 == 0, 8 <= d <= 16384; hidden 16-byte aligned, row and
+ * layer strides multiples of 8; m >= 0, n >= 0; n_layers <= 65535.
  * ---------------------------------------------------------------------- */
 typedef struct {
   const void *hidden;
   long long hidden_row_stride;
   int vis_start, m, text_start, n, d;
-  float *sim;             /* fp32 [m] out */
+  float *sim;             /* fp32 [m] out ([n_layers][sim_layer_stride] with several layers) */
   void *workspace;
   size_t workspace_bytes;
+  int n_layers;                   /* 0 or 1: one layer */
+  long long hidden_layer_stride;  /* elements, used when n_layers > 1 */
+  long long sim_layer_stride;     /* elements, >= m, used when n_layers > 1 */
 } pvlm_similarity_params;
 
 size_t pvlm_uvprune_similarity_workspace_bytes(const pvlm_similarity_params *p);

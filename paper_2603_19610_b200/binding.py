@@ -70,7 +70,8 @@ class AcceptParams(C.Structure):
 class SimilarityParams(C.Structure):
     _fields_ = [("hidden", C.c_void_p), ("hidden_row_stride", C.c_longlong),
                 ("vis_start", C.c_int), ("m", C.c_int), ("text_start", C.c_int), ("n", C.c_int), ("d", C.c_int),
-                ("sim", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+                ("sim", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("n_layers", C.c_int), ("hidden_layer_stride", C.c_longlong), ("sim_layer_stride", C.c_longlong)]
 
 
 class StepParams(C.Structure):
@@ -442,15 +443,22 @@ def accept_from_probs(p_tok, q_tok, uniforms):
 
 
 def uvprune_similarity(hidden, vis_start: int, m: int, text_start: int, n: int, *, out=None, workspace=None):
-    """sum_j cos(V_i, X_j) for the m visual rows of one layer's token representations
-    (see pvlm_uvprune_similarity).  hidden: bf16 [rows, d].  Returns fp32 [m]."""
+    """sum_j cos(V_i, X_j) for the m visual rows of a layer's token representations
+    (see pvlm_uvprune_similarity).  hidden: bf16 [rows, d] -> fp32 [m], or several layers at once,
+    bf16 [L, rows, d] -> fp32 [L, m] (one launch of each kernel for all of them)."""
     _need_cuda(hidden)
-    assert hidden.dtype == torch.bfloat16 and hidden.dim() == 2 and hidden.stride(1) == 1
-    sim = out if out is not None else torch.empty(m, dtype=torch.float32, device=hidden.device)
+    assert hidden.dtype == torch.bfloat16 and hidden.dim() in (2, 3) and hidden.stride(-1) == 1
+    layered = hidden.dim() == 3
+    L = hidden.shape[0] if layered else 1
+    shape = (L, m) if layered else (m,)
+    sim = out if out is not None else torch.empty(shape, dtype=torch.float32, device=hidden.device)
+    assert tuple(sim.shape) == shape and sim.stride(-1) == 1
     p = SimilarityParams()
-    p.hidden, p.hidden_row_stride = _ptr(hidden), hidden.stride(0)
-    p.vis_start, p.m, p.text_start, p.n, p.d = vis_start, m, text_start, n, hidden.shape[1]
+    p.hidden, p.hidden_row_stride = _ptr(hidden), hidden.stride(-2)
+    p.vis_start, p.m, p.text_start, p.n, p.d = vis_start, m, text_start, n, hidden.shape[-1]
     p.sim = _ptr(sim)
+    if layered:
+        p.n_layers, p.hidden_layer_stride, p.sim_layer_stride = L, hidden.stride(0), sim.stride(0)
     need = lib().pvlm_uvprune_similarity_workspace_bytes(C.byref(p))
     ws = workspace if workspace is not None else _workspace(hidden.device, "sim", need)
     p.workspace, p.workspace_bytes = _ptr(ws), ws.numel()

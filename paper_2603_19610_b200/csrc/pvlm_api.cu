@@ -187,7 +187,7 @@ static bool similarity_supported(const pvlm_similarity_params* p) {
 }
 
 size_t pvlm_uvprune_similarity_workspace_bytes(const pvlm_similarity_params* p) {
-  if (!p || p->m < 0 || p->n < 0 || !similarity_supported(p)) return 0;
+  if (!p || p->m < 0 || p->n < 0 || p->n_layers < 0 || p->n_layers > 65535 || !similarity_supported(p)) return 0;
   return similarity_workspace(*p);
 }
 
@@ -197,6 +197,9 @@ pvlm_status pvlm_uvprune_similarity(const pvlm_similarity_params* p, void* strea
   if (!similarity_supported(p)) return PVLM_ERR_UNSUPPORTED;
   if (!p->hidden || (p->m > 0 && !p->sim)) return PVLM_ERR_INVALID_ARG;
   if (!aligned(p->hidden, 16) || p->hidden_row_stride < p->d || p->hidden_row_stride % 8) return PVLM_ERR_INVALID_ARG;
+  if (p->n_layers < 0) return PVLM_ERR_INVALID_ARG;
+  if (p->n_layers > 65535) return PVLM_ERR_UNSUPPORTED;
+  if (p->n_layers > 1 && (p->hidden_layer_stride < 0 || p->hidden_layer_stride % 8 || p->sim_layer_stride < p->m)) return PVLM_ERR_INVALID_ARG;
   const pvlm_status w = check_ws(p->workspace, p->workspace_bytes, similarity_workspace(*p));
   if (w != PVLM_OK) return w;
   return launch_similarity(*p, (cudaStream_t)stream);

@@ -61,14 +61,30 @@ def test_zero_rows_and_strided_rows():
     assert e.value.status in (1, 2)
 
 
+def test_several_layers_in_one_call_equal_single_calls():
+    """Two and three layers through one call (one launch of each kernel for all of them): every layer's result is
+    bitwise what a call on that layer alone gives, and matches the oracle; a padded layer stride is honoured."""
+    rng = np.random.default_rng(41)
+    for L, m, n, d in [(2, 700, 90, 1024), (3, 33, 5, 64), (2, 1, 1, 8)]:
+        hb = [wl.f32_to_bf16_bits(rng.standard_normal((m + n + 3, d)).astype(np.float32) + (0.2 if l else 0.0)) for l in range(L)]
+        stack = torch.zeros((L, m + n + 7, d), dtype=torch.bfloat16, device="cuda")         # rows beyond the last are padding
+        for l in range(L):
+            stack[l, :m + n + 3] = bf16_cuda(hb[l])
+        sims = binding.uvprune_similarity(stack, 0, m, m, n)
+        torch.cuda.synchronize()
+        assert sims.shape == (L, m)
+        for l in range(L):
+            one, ref = check(hb[l], 0, m, m, n)
+            assert torch.equal(sims[l], one)
+
+
 @pytest.mark.parametrize("cid", [0, 1])
 def test_paper_uvprune_end_to_end(cid):
     """Eq. 1 -> Eq. 2 (layers 0 and 20) -> Eq. 3 -> gather, GPU against oracle."""
     cfg = wl.CONFIGS[cid]
     h0, hL = wl.hidden_layer(cfg, 0), wl.hidden_layer(cfg, 20)
     m, n = cfg.m, cfg.n_text
-    s0 = binding.uvprune_similarity(bf16_cuda(h0), 0, m, m, n)
-    sL = binding.uvprune_similarity(bf16_cuda(hL), 0, m, m, n)
+    s0, sL = binding.uvprune_similarity(torch.stack([bf16_cuda(h0), bf16_cuda(hL)]), 0, m, m, n)     # both end layers, one call
     _, k, v = wl.attn_layer(cfg, 0)
     kept, score, dk, dv = binding.uvprune_select_gather(sL, s0, 0, m, cfg.k_keep, bf16_cuda(k), bf16_cuda(v), want_score=True)
     torch.cuda.synchronize()
