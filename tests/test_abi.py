@@ -100,6 +100,23 @@ def test_workspace_queries_and_argument_errors_need_no_gpu():
     assert L.pvlm_uvprune_workspace_bytes(C.byref(u)) >= 400
     assert L.pvlm_uvprune_select_gather(C.byref(u), None) == 1          # no mass pointer
 
+    # similarity: the workspace grows with the layers of the call; bad layer counts and strides are refused before any launch
+    sm = binding.SimilarityParams()
+    sm.m, sm.n, sm.d, sm.hidden_row_stride = 1000, 100, 1024, 1024
+    one = L.pvlm_uvprune_similarity_workspace_bytes(C.byref(sm))
+    sm.n_layers = 2
+    assert one > 0 and L.pvlm_uvprune_similarity_workspace_bytes(C.byref(sm)) > one
+    sm.n_layers = -1
+    assert L.pvlm_uvprune_similarity_workspace_bytes(C.byref(sm)) == 0
+    sm.hidden = sm.sim = 4096
+    assert L.pvlm_uvprune_similarity(C.byref(sm), None) == 1
+    sm.n_layers, sm.hidden_layer_stride, sm.sim_layer_stride = 2, 1100 * 1024, 999
+    assert L.pvlm_uvprune_similarity(C.byref(sm), None) == 1            # the layers' outputs would overlap
+    sm.hidden_layer_stride, sm.sim_layer_stride = 1100 * 1024 + 4, 1000
+    assert L.pvlm_uvprune_similarity(C.byref(sm), None) == 1            # layer stride not a multiple of 8 elements
+    sm.hidden_layer_stride = 1100 * 1024
+    assert L.pvlm_uvprune_similarity(C.byref(sm), None) == 3            # no workspace
+
     # the decision-only entry points
     assert L.pvlm_select_from_scores(None, 100, 101, None, None, 0, None) == 1    # k > m
     assert L.pvlm_select_from_scores(None, 100, 10, None, None, 0, None) == 1     # no scores

@@ -78,6 +78,25 @@ def test_several_layers_in_one_call_equal_single_calls():
             assert torch.equal(sims[l], one)
 
 
+def test_several_layers_with_offsets_and_strided_views():
+    """Layers that are views of a larger buffer (padded row stride, layer stride larger than a layer, rows before the
+    visual span and between the spans), results into a strided output: each layer against the oracle."""
+    rng = np.random.default_rng(43)
+    L, v0, m, gap, n, d = 2, 5, 300, 4, 37, 192
+    rows = v0 + m + gap + n + 2
+    big = torch.zeros((L, rows + 9, d + 16), dtype=torch.bfloat16, device="cuda")
+    hb = [wl.f32_to_bf16_bits(rng.standard_normal((rows, d)).astype(np.float32)) for _ in range(L)]
+    for l in range(L):
+        big[l, :rows, :d] = bf16_cuda(hb[l])
+    out = torch.full((L, m + 11), -7.0, dtype=torch.float32, device="cuda")
+    sims = binding.uvprune_similarity(big[:, :rows, :d], v0, m, v0 + m + gap, n, out=out[:, :m])
+    torch.cuda.synchronize()
+    assert (out[:, m:] == -7.0).all()                                     # nothing written past a layer's m results
+    for l in range(L):
+        one, ref = check(hb[l], v0, m, v0 + m + gap, n)
+        assert torch.equal(sims[l], one)
+
+
 @pytest.mark.parametrize("cid", [0, 1])
 def test_paper_uvprune_end_to_end(cid):
     """Eq. 1 -> Eq. 2 (layers 0 and 20) -> Eq. 3 -> gather, GPU against oracle."""
