@@ -218,6 +218,15 @@ def test_head_dim_64_on_the_tensor_core_path(pvlm_option):
     assert_o_close(o[1], O1)
 
 
+@pytest.mark.parametrize("Hq,R", [(16, 11), (16, 16), (14, 15)])
+def test_head_dim_64_with_wide_row_groups(Hq, R, pvlm_option):
+    """D = 64 together with 88 / 128 rows per KV head (split-column mode) and 105 rows (alternate tiles, 3 ring slots)."""
+    pvlm_option("attn_max_ctas", 4)
+    n_ctx = 1700
+    qb, kb, vb = wl.make_qkv(Hq, 2, 64, R, n_ctx + R, sink=True, seed=640 + R)
+    run_case(qb, kb, vb, n_ctx)
+
+
 def test_head_major_cache_layout():
     """K/V stored [Hkv][T][D] and passed through the strides."""
     Hq, Hkv, D, n_ctx, R = 16, 4, 128, 900, 7
