@@ -305,6 +305,15 @@ def run_ours(args):
     wall_end = time.time()
     total_ms = t0.elapsed_time(t1)
     clocks = sampler.stop(wall_begin, wall_end) if sampler else None
+    # host time to queue one step, measured while the stream is held busy by a spin kernel (the calls only queue): the
+    # step is GPU-bound where this is well below the step time, launch-bound where it is not (the one-layer configs)
+    with torch.cuda.stream(main_stream):
+        torch.cuda._sleep(int(1e8))
+        hq0 = time.perf_counter()
+        for _ in range(20):
+            device_step() if args.serial_step else fused_step()
+        host_enqueue_us = (time.perf_counter() - hq0) * 1e6 / 20
+        barrier()
     # ---- sustained figure: the SAME step for at least two more seconds (the driver-sized region above is a burst: a few
     # tenths of a second, before the board settles at its power cap); reported beside the burst figures, never instead.
     sustained = None
@@ -411,6 +420,7 @@ def run_ours(args):
         "gpu_launches": args.steps * (7 if args.serial_step else 8),
         "stages_note": "stage times come from a separate pass that runs the stages as three serial calls; the timed step is one "
                        "call in which the accept stage and the selection-independent part of the gather run on a second stream",
+        "host_enqueue_us_per_step": host_enqueue_us,
         "stages_us": {"attention": attn_avg_ms * 1e3, "prune_select_gather": sum(prune_ms) / len(prune_ms) * 1e3,
                       "softmax_accept": sum(acc_ms) / len(acc_ms) * 1e3},
         "step_gbs": (ab_attn + ab_prune + ab_acc) / (ms_per_step * 1e-3) / 1e9,
