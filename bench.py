@@ -234,6 +234,10 @@ def run_ours(args):
         e.record()                                  # forces creation of the underlying cudaEvent_t
     torch.cuda.synchronize()
     pa.prof_event_begin, pa.prof_event_end = k_ev[0].cuda_event, k_ev[1].cuda_event
+    # the same block without the two timing events, for the steps whose kernel time is not sampled (every event is one
+    # more stream operation for the host to queue, which shows at the one-layer configs)
+    pa_plain = type(pa).from_buffer_copy(pa)
+    pa_plain.prof_event_begin = pa_plain.prof_event_end = None
     main_kernel_ms = []
     pp = binding.prune_params(mass_cur, mass_ref, 0, cfg.m, cfg.k_keep, kept, None, src_k, src_v, dK, dV)
     pc = binding.accept_params(tl, dl, tok, u, 1.0, outs)
@@ -277,8 +281,15 @@ def run_ours(args):
         e.record()
     torch.cuda.synchronize()
 
-    def fused_step():
-        binding.verify_step(pa, pp, pc, device=dev, overlap=(copy_stream, ov_ev[0], ov_ev[1]))
+    prepared = {}
+
+    def fused_step(sampled=True):
+        sp = prepared.get(sampled)
+        if sp is None:                                   # marshalled once per variant, then only re-queued
+            prepared[sampled] = binding.verify_step(pa if sampled else pa_plain, pp, pc, device=dev,
+                                                    overlap=(copy_stream, ov_ev[0], ov_ev[1]))
+        else:
+            binding.verify_step_again(sp, dev)
 
     sampler = ClockSampler(local_rank) if rank == 0 else None     # started early: nvidia-smi takes a while to deliver
     # The step runs on a high-priority stream, so that the small kernels of its critical chain (combine, mass, select)
@@ -293,11 +304,12 @@ def run_ours(args):
         t0, t1 = ev(), ev()
         t0.record()
         for i in range(args.steps):
+            sampled = i % 8 == 7 or i == args.steps - 1
             if args.serial_step:
                 device_step()                            # the three stages as serial calls on one stream
             else:
-                fused_step()                             # ONE call per step: all stages, inputs resident in HBM
-            if i % 8 == 7 or i == args.steps - 1:       # sample the in-library kernel events (needs a sync: every 8th step)
+                fused_step(sampled)                      # ONE call per step: all stages, inputs resident in HBM
+            if sampled:                                  # read the in-library kernel events (needs a sync: every 8th step)
                 k_ev[1].synchronize()
                 main_kernel_ms.append(k_ev[0].elapsed_time(k_ev[1]))
         t1.record()
@@ -311,7 +323,7 @@ def run_ours(args):
         torch.cuda._sleep(int(1e8))
         hq0 = time.perf_counter()
         for _ in range(20):
-            device_step() if args.serial_step else fused_step()
+            device_step() if args.serial_step else fused_step(False)
         host_enqueue_us = (time.perf_counter() - hq0) * 1e6 / 20
         barrier()
     # ---- sustained figure: the SAME step for at least two more seconds (the driver-sized region above is a burst: a few
@@ -329,7 +341,7 @@ def run_ours(args):
             s0, s1 = ev(), ev()
             s0.record()
             for i in range(n_sus):
-                device_step() if args.serial_step else fused_step()
+                device_step() if args.serial_step else fused_step(i % 64 == 63 or i == n_sus - 1)
                 if i % 64 == 63 or i == n_sus - 1:
                     k_ev[1].synchronize()
                     sus_kernel_ms.append(k_ev[0].elapsed_time(k_ev[1]))
@@ -376,7 +388,7 @@ def run_ours(args):
     if world == 1 and not args.no_draft_stream:
         saved = (pa.prof_event_begin, pa.prof_event_end)
         pa.prof_event_begin = pa.prof_event_end = None          # timing events cannot be read back from a captured launch
-        graph_report = graph_replay_leg(torch, dev, device_step, fused_step, min(args.steps, 50))
+        graph_report = graph_replay_leg(torch, dev, device_step, lambda: fused_step(False), min(args.steps, 50))
         pa.prof_event_begin, pa.prof_event_end = saved
     draft_report = None
     if world == 1 and not args.no_draft_stream:

@@ -131,7 +131,8 @@ pvlm_status pvlm_verify_attn(const pvlm_attn_params *p, void *stream);
 /* Health check of the last pvlm_verify_attn issued with this parameter block (same workspace):
  * every wait inside the kernels is bounded, and one that expires records it in the workspace
  * instead of hanging.  This call SYNCHRONISES `stream`, reads that word and returns PVLM_OK or
- * PVLM_ERR_TIMEOUT.  Optional: results of a call that timed out are undefined either way. */
+ * PVLM_ERR_TIMEOUT.  Optional: results of a call that timed out are undefined either way.
+ * (The word is cleared by the call's first kernel, so it always describes the last call.) */
 pvlm_status pvlm_verify_attn_check(const pvlm_attn_params *p, void *stream);
 
 /* ------------------------------------------------------------------------

@@ -394,6 +394,15 @@ def verify_step(attn: AttnParams | None, prune: PruneParams | None, accept: Acce
     return sp
 
 
+def verify_step_again(sp: StepParams, device=None) -> None:
+    """Queue the step of a parameter block that verify_step returned once more (same buffers, same stages): the
+    marshalling is done once, a repeated step costs the C call alone."""
+    dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+    st = lib().pvlm_verify_step(C.byref(sp), _stream(dev))
+    if st != 0:
+        raise PvlmError(st, "pvlm_verify_step")
+
+
 def uvprune_select_static(mass_cur, mass_ref, vis_start: int, m: int, k: int, kept_idx, score=None):
     """Top-K selection through pvlm_uvprune_select_static, the entry point for callers that
     cannot allocate device memory: the library's built-in key buffer is the only scratch and

@@ -294,9 +294,15 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     if (vp != PVLM_OK) return vp;
   }
   // ---- host -> device: this step's inputs ----
-  if (overlap) {                       // the copy stream starts after whatever is already queued on `stream`
+  // The side stream is forked from `stream` (an event recorded there, a wait on the side) only at the first point where
+  // something is queued on it, and joined back at the end if it was forked: a call with nothing for it costs no
+  // stream operation, and a stream capture of the call always closes.
+  bool forked = false;
+  const bool side_uploads = p->run_accept && (p->h_target_logits || p->h_draft_logits || p->h_draft_tokens || p->h_uniforms);
+  if (overlap && side_uploads) {       // the copies start after whatever is already queued on `stream`
     e = cudaEventRecord(ea, s);
     if (ok()) e = cudaStreamWaitEvent(cs, ea, 0);
+    forked = true;
   }
   if (p->run_attn) {
     const size_t q_layer = (size_t)a.R * a.Hq * a.D * 2;
@@ -326,7 +332,7 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
                               cudaMemcpyHostToDevice, s);
     }
   }
-  if (overlap && p->run_attn && (p->h_q || p->h_k_window || p->h_v_window) && ok()) {
+  if (overlap && side_uploads && p->run_attn && (p->h_q || p->h_k_window || p->h_v_window) && ok()) {
     // the attention's own inputs go first over the link: the accept inputs, needed much later, queue behind them
     e = cudaEventRecord(eb, s);
     if (ok()) e = cudaStreamWaitEvent(cs, eb, 0);
@@ -361,7 +367,10 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
   } else if (accept_on_side || split_gather) {
     e = cudaEventRecord(eb, s);
   }
-  if ((accept_on_side || split_gather) && ok()) e = cudaStreamWaitEvent(cs, eb, 0);
+  if ((accept_on_side || split_gather) && ok()) {
+    e = cudaStreamWaitEvent(cs, eb, 0);
+    forked = true;
+  }
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   if (split_gather && (st = launch_uvprune_parts(p->prune, false, 1, cs)) != PVLM_OK) return st;
   if (accept_on_side) {
@@ -377,6 +386,7 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     if (overlap) {
       e = cudaEventRecord(eb, s);
       if (ok()) e = cudaStreamWaitEvent(cs, eb, 0);
+      forked = true;
     }
     if (ok()) e = cudaMemcpy2DAsync(p->h_o, q_layer, a.o, (size_t)a.q_layer_stride * 2, q_layer, a.n_layers, cudaMemcpyDeviceToHost, cs);
     if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
@@ -399,10 +409,10 @@ pvlm_status pvlm_verify_step(const pvlm_step_params* p, void* stream) {
     e = cudaMemcpyAsync(p->h_n_accept, c.n_accept, (size_t)c.batch * 4, cudaMemcpyDeviceToHost, s);
   if (p->run_accept && !accept_on_side && p->h_out_tokens && ok())
     e = cudaMemcpyAsync(p->h_out_tokens, c.out_tokens, (size_t)c.batch * (c.gamma + 1) * 4, cudaMemcpyDeviceToHost, s);
-  // The side stream was forked from `stream` at the top; whatever was (or was not) queued on it, it is joined back
-  // here, so that synchronising `stream` alone covers everything and a stream capture of the call always closes.
-  if (overlap && ok()) e = cudaEventRecord(ea, cs);
-  if (overlap && ok()) e = cudaStreamWaitEvent(s, ea, 0);
+  // A forked side stream is joined back here, so that synchronising `stream` alone covers everything and a stream
+  // capture of the call closes.
+  if (overlap && forked && ok()) e = cudaEventRecord(ea, cs);
+  if (overlap && forked && ok()) e = cudaStreamWaitEvent(s, ea, 0);
   if (!ok()) { set_cuda_error((int)e); return PVLM_ERR_CUDA; }
   return PVLM_OK;
 }

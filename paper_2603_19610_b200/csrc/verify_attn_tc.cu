@@ -32,6 +32,8 @@
 // reuses m; otherwise (and on the first tile of a segment) all softmax threads take a slow path that
 // reduces the tile's row maxima, rescales the running sums and the TMEM accumulator, and goes on.
 // Every mbarrier wait is bounded: on expiry the CTA sets a status word and leaves cleanly.
+#include <atomic>
+
 #include "pvlm_common.cuh"
 
 #include <cuda.h>
@@ -284,6 +286,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   auto bar = [&](int i) { return smem_addr(bars + i); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // The call's status word is cleared here instead of by a memset in front of the launch (one stream operation less per
+  // call).  A CTA reports an expired wait at its teardown, at least kWaitLimitNs after it started, and CTA 0 is the
+  // first CTA of the grid to be dispatched, so this store comes before any report of this call.
+  if (blockIdx.x == 0 && tid == 0) *a.status = 0;
 
   // ---- this CTA's range of the flattened tile sequence ----
   const long long W = a.total_tiles;
@@ -1280,6 +1286,20 @@ bool make_kv_map(CUtensorMap* map, const void* base, const pvlm_attn_params& p, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// cudaFuncSetAttribute once per kernel and device instead of on every launch (the attribute belongs to the device's
+// copy of the function; devices beyond the 64th set it every time).  The kernel is a template argument, so that every
+// instantiation has a flag word of its own.
+template <auto Kernel>
+void set_max_dynamic_smem_once(int bytes) {
+  static std::atomic<unsigned long long> done{0};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  const unsigned long long bit = (dev >= 0 && dev < 64) ? 1ull << dev : 0ull;
+  if (bit && (done.load(std::memory_order_acquire) & bit)) return;
+  cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (bit) done.fetch_or(bit, std::memory_order_release);
+}
+
 template <int NRP>
 constexpr int tc_smem_bytes() {
   return 1024 /*alignment slack*/ + ring_slots(NRP) * kTileBytes + 2 * NRP * 128 + 2 * NRP * 256 + 3 * 256 * 4 + 32 * 8 + 64;
@@ -1290,13 +1310,13 @@ void launch_tc(const CUtensorMap& mk, const CUtensorMap& mv, const TcArgs& a, cu
   constexpr int smem = tc_smem_bytes<NRP>();
   if constexpr (!split_cols(NRP)) {
     if (a.rows <= NRP - 8) {
-      cudaFuncSetAttribute(attn_tc_kernel<NRP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      set_max_dynamic_smem_once<attn_tc_kernel<NRP, true>>(smem);
       attn_tc_kernel<NRP, true><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
       return;
     }
   }
   {
-    cudaFuncSetAttribute(attn_tc_kernel<NRP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    set_max_dynamic_smem_once<attn_tc_kernel<NRP, false>>(smem);
     attn_tc_kernel<NRP, false><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
   }
 }
@@ -1304,7 +1324,7 @@ void launch_tc(const CUtensorMap& mk, const CUtensorMap& mv, const TcArgs& a, cu
 template <int NRP>
 void launch_tc_mass(const CUtensorMap& mk, const TcMassArgs& a, cudaStream_t s) {
   constexpr int smem = 1024 + kMassKStages * kTileBytes + 2 * NRP * 128 + 128 * 4 + 24 * 8 + 64;
-  cudaFuncSetAttribute(attn_tc_mass_kernel<NRP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  set_max_dynamic_smem_once<attn_tc_mass_kernel<NRP>>(smem);
   const cudaError_t e = launch_dependent(attn_tc_mass_kernel<NRP>, dim3(a.n_cta), dim3(kThreads), smem, s, mk, a);
   if (e != cudaSuccess) set_cuda_error((int)e);
 }
@@ -1395,7 +1415,6 @@ pvlm_status launch_verify_attn_tc(const pvlm_attn_params& p, const AttnTcPlan& p
     // worth it only where the mass pass re-reads a sizeable share of what this launch streams: every layer's mass wanted
     a.l2_hints = (p.mass != nullptr && (p.mass_layers == nullptr || p.n_mass_layers == p.n_layers)) ? 1 : 0;
   }
-  cudaMemsetAsync(a.status, 0, 4, s);
   if (p.prof_event_begin) cudaEventRecord((cudaEvent_t)p.prof_event_begin, s);
   switch (plan.nrp) {
     case 16: launch_tc<16>(mk, mv, a, s); break;
