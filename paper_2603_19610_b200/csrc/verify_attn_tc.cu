@@ -286,10 +286,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   auto bar = [&](int i) { return smem_addr(bars + i); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // The call's status word is cleared here instead of by a memset in front of the launch (one stream operation less per
-  // call).  A CTA reports an expired wait at its teardown, at least kWaitLimitNs after it started, and CTA 0 is the
-  // first CTA of the grid to be dispatched, so this store comes before any report of this call.
-  if (blockIdx.x == 0 && tid == 0) *a.status = 0;
 
   // ---- this CTA's range of the flattened tile sequence ----
   const long long W = a.total_tiles;
@@ -320,6 +316,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  // The launch is a programmatic dependent of whatever kernel precedes it in the stream (the merge of the previous decode
+  // step, the gather of the previous round): the set-up above overlaps that kernel's tail; everything below reads
+  // tensors it may have produced (Q, K, V) or writes a workspace it may still read, so it comes after this wait.
+  pdl_wait();
+  // The call's status word is cleared here instead of by a memset in front of the launch (one stream operation less per
+  // call, and nothing between this launch and the kernel before it).  A CTA reports an expired wait at its teardown, at
+  // least kWaitLimitNs after it started, and CTA 0 is the first CTA of the grid to be dispatched, so this store comes
+  // before any report of this call.
+  if (blockIdx.x == 0 && tid == 0) *a.status = 0;
   const uint32_t tmem_O = tmem;                    // O accumulators of the two softmax groups: columns [g*NRP, (g+1)*NRP)
   const uint32_t tmem_S = tmem + (SC ? 1 : 2) * NRP;   // score buffers (split-column mode has one accumulator)
 
@@ -1311,13 +1316,15 @@ void launch_tc(const CUtensorMap& mk, const CUtensorMap& mv, const TcArgs& a, cu
   if constexpr (!split_cols(NRP)) {
     if (a.rows <= NRP - 8) {
       set_max_dynamic_smem_once<attn_tc_kernel<NRP, true>>(smem);
-      attn_tc_kernel<NRP, true><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
+      const cudaError_t e = launch_dependent(attn_tc_kernel<NRP, true>, dim3(a.n_cta), dim3(kThreads), smem, s, mk, mv, a);
+      if (e != cudaSuccess) set_cuda_error((int)e);
       return;
     }
   }
   {
     set_max_dynamic_smem_once<attn_tc_kernel<NRP, false>>(smem);
-    attn_tc_kernel<NRP, false><<<a.n_cta, kThreads, smem, s>>>(mk, mv, a);
+    const cudaError_t e = launch_dependent(attn_tc_kernel<NRP, false>, dim3(a.n_cta), dim3(kThreads), smem, s, mk, mv, a);
+    if (e != cudaSuccess) set_cuda_error((int)e);
   }
 }
 
