@@ -262,7 +262,7 @@ uvprune_select_cluster_kernel(const SelArgs a) {
                                                          // that one cluster barrier per pass is enough (see below)
   __shared__ unsigned int hist_l[256 * 32];
   __shared__ unsigned int s_prefix, s_remaining;
-  __shared__ int s_cnt[2];                               // (greater, equal) counts of this CTA (read remotely)
+  __shared__ int s_cnt[kSelCluster];                     // (greater << 16 | equal) counts of every CTA, each written by its owner
   __shared__ int wsum[33];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int base = (int)rank * (ITEMS * kSelThreads) + warp * (ITEMS * 32) + lane;
@@ -337,22 +337,27 @@ uvprune_select_cluster_kernel(const SelArgs a) {
     warp_eq += __popc(__ballot_sync(0xffffffffu, vld && key[i] == tau));
     warp_gt += __popc(__ballot_sync(0xffffffffu, vld && key[i] > tau));
   }
-  int cta_eq, cta_gt;
-  int eq_run = block_exclusive_scan(lane == 31 ? warp_eq : 0, wsum, cta_eq);
-  eq_run = __shfl_sync(0xffffffffu, eq_run, 31);
-  block_exclusive_scan(lane == 31 ? warp_gt : 0, wsum, cta_gt);
-  if (tid == 0) { s_cnt[0] = cta_gt; s_cnt[1] = cta_eq; }
+  // one scan for both counts: a CTA holds at most ITEMS * 1024 <= 32768 keys, so (greater, equal) fit the halves of a word
+  static_assert(ITEMS * kSelThreads <= 32768, "packed counts");
+  int cta_cnt;
+  int run = block_exclusive_scan(lane == 31 ? ((warp_gt << 16) | warp_eq) : 0, wsum, cta_cnt);
+  int eq_run = __shfl_sync(0xffffffffu, run, 31) & 0xFFFF;
+  // every CTA stores its counts into every member's shared memory (distributed shared memory), so that after ONE cluster
+  // barrier all reads are local and nobody's shared memory is touched again
+  if (tid < kSelCluster) *cluster.map_shared_rank(&s_cnt[rank], tid) = cta_cnt;
   cluster.sync();
   // counts of the CTAs before this one: equals before => how many of mine are kept; kept before => output offset
   int eq_base = 0, sel_base = 0;
-  for (unsigned r = 0; r < rank; ++r) {
-    const int* c = cluster.map_shared_rank(s_cnt, r);
-    const int g = c[0], e = c[1];
-    const int kept_eq = min(max(take_eq - eq_base, 0), e);
-    sel_base += g + kept_eq;
-    eq_base += e;
+#pragma unroll
+  for (int r = 0; r < kSelCluster; ++r) {
+    if (r < (int)rank) {
+      const unsigned c = (unsigned)s_cnt[r];
+      const int g = (int)(c >> 16), e = (int)(c & 0xFFFFu);
+      const int kept_eq = min(max(take_eq - eq_base, 0), e);
+      sel_base += g + kept_eq;
+      eq_base += e;
+    }
   }
-  cluster.sync();                                        // nobody leaves while its counts may still be read
   eq_run += eq_base;
   uint32_t selbits = 0u;
   int warp_sel = 0;
