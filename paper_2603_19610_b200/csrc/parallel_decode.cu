@@ -42,9 +42,14 @@ void accept_block(const pvlm_decode_params& p, int gamma, int batch, pvlm_accept
 bool make_layout(const pvlm_decode_params& p, DecodeLayout& l) {
   pvlm_accept_params c;
   AcceptPlan plan;
-  accept_block(p, p.gamma, 1, c);
-  if (!make_accept_plan(c, plan)) return false;
-  l.accept_ws = align_up(plan.total, 256);
+  // A round verifies between 1 and gamma tokens, and a SHORTER window can need more scratch (fewer logit rows are cut
+  // into more statistics chunks each): size for the largest of them.
+  l.accept_ws = 0;
+  for (int nv = 1; nv <= p.gamma; ++nv) {
+    accept_block(p, nv, 1, c);
+    if (!make_accept_plan(c, plan)) return false;
+    if (align_up(plan.total, 256) > l.accept_ws) l.accept_ws = align_up(plan.total, 256);
+  }
   accept_block(p, 0, p.gamma, c);
   if (!make_accept_plan(c, plan)) return false;
   l.sample_ws = align_up(plan.total, 256);

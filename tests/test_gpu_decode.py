@@ -35,7 +35,10 @@ def log_rows(log):
 @pytest.mark.parametrize("V,K,gamma,sigma,seed", [(50, 40, 4, 0.8, 3), (1000, 64, 9, 0.5, 7), (4099, 33, 1, 0.7, 11),
                                                    (32000, 24, 5, 0.3, 5), (17, 80, 12, 1.5, 9), (152064, 12, 3, 0.4, 2),
                                                    (300, 200, 64, 0.05, 1), (300, 200, 64, 0.6, 2),      # the widest window
-                                                   (1000, 500, 33, 0.2, 3), (5, 1000, 2, 0.3, 4)])       # long runs
+                                                   (1000, 500, 33, 0.2, 3), (5, 1000, 2, 0.3, 4),        # long runs
+                                                   # windows whose gamma - 1 pending drafts need MORE accept scratch than
+                                                   # the full window (fewer rows, more statistics chunks per row)
+                                                   (152064, 16, 7, 0.1, 6), (50000, 16, 13, 0.1, 8), (16384, 20, 13, 0.1, 9)])
 def test_tokens_and_round_log_match_the_oracle(V, K, gamma, sigma, seed):
     tl, dl, ud, ua, ur = make_case(V, K, gamma, sigma, seed)
     ref = oracle_decode(tl, dl, gamma, K, ud, ua, ur)
