@@ -27,6 +27,27 @@ def gpu_decode(tl, dl, gamma, K, ud, ua, ur, **kw):
     return binding.parallel_decode(d(tl), d(dl), gamma, K, d(ud), d(ua), d(ur), **kw)
 
 
+def first_token_mismatch_is_a_rounding_band_event(gpu_tokens, ref_tokens, tl, dl, ud, ua, ur, temperature=1.0):
+    """Where the library's tokens leave the oracle's, the FIRST differing token must be a draw whose u * Z lies within
+    1e-5 * Z of the step of the cumulative weights between the two tokens, with no weight between them (the documented
+    band of the fp32-weight / fp64-sum inverse CDF against the fp64 oracle); what follows such a draw may differ freely.
+    The weights are those of the position's three possible draws: the draft's q, the residual max(0, p - q), the target's p."""
+    from oracle.accept import softmax64
+    n = min(len(gpu_tokens), len(ref_tokens))
+    bad = np.nonzero(np.asarray(gpu_tokens[:n]) != np.asarray(ref_tokens[:n]))[0]
+    assert len(bad) > 0
+    i = int(bad[0])
+    a, b = sorted((int(gpu_tokens[i]), int(ref_tokens[i])))
+    p = softmax64(np.asarray(tl)[i], temperature)
+    q = softmax64(np.asarray(dl)[i], temperature)
+    us = np.concatenate([np.asarray(x, dtype=np.float64).ravel() for x in (ud, ua, ur)])
+    for w in (q, np.maximum(0.0, p - q), p):
+        c = np.cumsum(w)
+        if w[a + 1:b].sum() == 0.0 and np.abs(us * c[-1] - c[a]).min() <= 1e-5 * c[-1]:
+            return True
+    return False
+
+
 def log_rows(log):
     return [[r["mode"], r["verified"], r["accepted"], r["emitted"], r["dropped"], r["start"],
              r["target_ctx"], r["draft_ctx"], r["draft_keep"]] for r in log]

@@ -14,7 +14,7 @@ from oracle.uvprune import gather_rows, score_fp32, select_topk
 from paper_2603_19610_b200 import binding, workloads as wl
 from helpers import assert_o_close, assert_rel_close, bits_of
 from test_gpu_accept import check_against_oracle
-from test_gpu_decode import gpu_decode, log_rows, make_case
+from test_gpu_decode import first_token_mismatch_is_a_rounding_band_event, gpu_decode, log_rows, make_case
 from test_gpu_prune import gpu_select
 from test_gpu_rate import run_case as rate_case
 from test_gpu_similarity import check as similarity_check
@@ -174,7 +174,11 @@ def test_step_overlap_mode_random_gather_splits():
 
 
 def test_parallel_decode_random_windows_vocabularies_and_temperatures():
+    """Tokens, round count and round log equal the oracle's.  A draw that lands within the rounding band of a step of
+    the cumulative weights (about one in 1e4 cases; none among the default 60) may give the neighbouring token, after
+    which the two runs differ legitimately: such a case is checked to be exactly that, and at most one in 500 may be."""
     rng = np.random.default_rng(2)
+    banded = 0
     for case in range(CASES):
         V = int(rng.choice([2, 3, 17, 50, 257, 1000, 4099, int(rng.integers(2, 20000))]))
         K, gamma = int(rng.integers(1, 60)), int(rng.integers(1, 17))
@@ -185,9 +189,14 @@ def test_parallel_decode_random_windows_vocabularies_and_temperatures():
         for serial in (False, True):
             out = gpu_decode(tl, dl, gamma, K, ud, ua, ur, serial=serial, temperature=temp)
             tag = (case, V, K, gamma, sigma, temp, serial)
-            assert out["rounds"] == ref["rounds"], tag
-            assert out["log"].tolist() == log_rows(ref["log"]), tag
-            assert (out["tokens"].numpy() == ref["tokens"]).all(), tag
+            got = out["tokens"].numpy()
+            if len(got) == len(ref["tokens"]) and (got == ref["tokens"]).all():
+                assert out["rounds"] == ref["rounds"], tag
+                assert out["log"].tolist() == log_rows(ref["log"]), tag
+            else:
+                assert first_token_mismatch_is_a_rounding_band_event(got, ref["tokens"], tl, dl, ud, ua, ur, temp), tag
+                banded += 1
+    assert banded <= max(1, 2 * CASES // 500), banded
 
 
 def test_acceptance_rate_random_sizes_and_strides():
