@@ -219,4 +219,14 @@ def test_similarity_random_shapes():
         h[v0 + m:] += 0.3                                # text rows share a direction
         if m > 2 and rng.integers(0, 4) == 0:
             h[v0 + 1] = 0                                # a zero visual row
-        similarity_check(wl.f32_to_bf16_bits(h), v0, m, v0 + m, n)
+        hb = wl.f32_to_bf16_bits(h)
+        one, _ = similarity_check(hb, v0, m, v0 + m, n)
+        if case % 3 == 0:                                # the same layer inside a two- or three-layer call: bitwise the same result
+            L = 2 + case % 2
+            stack = torch.zeros((L, h.shape[0] + int(rng.integers(0, 4)), d), dtype=torch.bfloat16, device="cuda")
+            for l in range(L):
+                other = wl.f32_to_bf16_bits(rng.standard_normal(h.shape).astype(np.float32))
+                stack[l, :h.shape[0]] = torch.from_numpy((hb if l == L - 1 else other).view(np.int16)).view(torch.bfloat16).cuda()
+            sims = binding.uvprune_similarity(stack, v0, m, v0 + m, n)
+            torch.cuda.synchronize()
+            assert torch.equal(sims[L - 1], one), (case, m, n, d, v0, L)
